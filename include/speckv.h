@@ -322,6 +322,23 @@ int speckv_get_status(speckv_ctx *ctx, speckv_status *out, void *stream);
 int speckv_get_stats(speckv_ctx *ctx, speckv_stats *out, void *stream);
 int speckv_clear_status(speckv_ctx *ctx, void *stream); /* status and counters; asynchronous */
 
+/* Every wait inside the kernels is bounded (the engine's failure mode "a request that never completes"
+ * must come back as a status, never as a kernel that does not end): the compressor's scan polls the
+ * sizes of earlier tiles at most lookback_polls times per window of 64 tiles (>= 200 ns per poll), and
+ * a warp waits at most wait_ns nanoseconds on a shared-memory barrier.  A wait that runs out is counted
+ * as SPECKV_ST_TIMEOUT (index = first page of the tile whose place in the log could not be computed,
+ * or 0xFFFFFFF0..0xFFFFFFF3 for a barrier wait of an encoder, a record stage, the loader, the scanner);
+ * the tiles behind it in list order are not placed, their page-table entries and the cursor stay as they
+ * were, and the call still ends.  Defaults: 4,194,304 polls and 2 s; 0 selects the default.  Host-side
+ * setting of the context, applies to later speckv_compress calls.  No counterpart in the paper. */
+int speckv_set_wait_limits(speckv_ctx *ctx, uint32_t lookback_polls, uint64_t wait_ns);
+
+/* Fault injection for tests of those limits, made on the host: the next speckv_compress call (only)
+ * never hands out its first n_tiles tiles of 20 pages, as if the CTAs that drew them had stalled.
+ * Every later tile then waits for sizes that are never published, until its limit runs out.  Nothing
+ * faults or traps; combine with short limits.  n_tiles = 0 cancels. */
+int speckv_inject_missing_tiles(speckv_ctx *ctx, uint32_t n_tiles);
+
 /* Introspection for tools and tests.  Device pointers stay owned by the context. */
 void *speckv_pool_ptr(speckv_ctx *ctx);       /* uint8  [pool_bytes]                       */
 void *speckv_pte_ptr(speckv_ctx *ctx);        /* uint64 [n_layers*blocks_per_layer*2*H]    */

@@ -40,18 +40,33 @@ __device__ __forceinline__ unsigned long long global_ns()
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait for the phase with the given parity: gives up after kWaitNs nanoseconds (or
-// kWaitLimit polls), or as soon as `abort` (shared memory) becomes non-zero.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int *abort = nullptr)
+// Bounded wait for the phase with the given parity: gives up after limit_ns nanoseconds (or
+// kWaitLimit polls), or as soon as `abort` (shared memory) becomes non-zero.  Each lane decides for
+// itself: use it where a subset of lanes waits on barriers of their own.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int *abort = nullptr,
+                                          unsigned long long limit_ns = kWaitNs)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
     for (uint32_t i = 0; i < kWaitLimit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if (abort && *abort) return false;
-        if ((i & 63u) == 63u && global_ns() - t0 > kWaitNs) return false;
+        if ((i & 63u) == 63u && global_ns() - t0 > limit_ns) return false;
     }
     return false;
+}
+// The same wait made by all 32 lanes of a warp, with one answer for the whole warp: lanes that gave up
+// in the same instant in which others saw the phase complete look once more (a completed phase stays
+// complete until this warp moves on), so the warp never splits into lanes that leave and lanes that stay.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, const volatile int *abort = nullptr,
+                                               unsigned long long limit_ns = kWaitNs)
+{
+    bool ok = mbar_try_wait(bar, parity);
+    if (__all_sync(0xFFFFFFFFu, ok)) return true;
+    if (!ok) ok = mbar_wait(bar, parity, abort, limit_ns);
+    if (__all_sync(0xFFFFFFFFu, ok)) return true;
+    if (!ok) ok = mbar_try_wait(bar, parity);
+    return __all_sync(0xFFFFFFFFu, ok);
 }
 // bulk asynchronous copy global -> shared (bytes multiple of 16; both addresses 16-byte aligned);
 // completion is signalled on the mbarrier as transaction bytes

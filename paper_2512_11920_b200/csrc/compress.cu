@@ -398,7 +398,7 @@ __global__ void __launch_bounds__(kCThreads, 1) compress_kernel(CompressArgs a)
         const uint4 *in = reinterpret_cast<const uint4 *>(smem + kOffIn) + warp * (kPageBytes / 16);
         for (uint32_t j = 0;; ++j) {
             const uint32_t rs = j % kRecStages, rpar = (j / kRecStages) & 1u;
-            if (!mbar_wait(bar_in_full(warp), j & 1u, s_abort)) { give_up(0xFFFFFFF0u); return; }
+            if (!mbar_wait_warp(bar_in_full(warp), j & 1u, s_abort, a.wait_ns)) { give_up(0xFFFFFFF0u); return; }
             // read now: the loader reuses these words as soon as the page buffers are released
             const bool done = s_info[kEnc] != 0u, live = s_info[warp] != 0u;
             const uint32_t tile = s_info[kEnc + 1];
@@ -411,7 +411,7 @@ __global__ void __launch_bounds__(kCThreads, 1) compress_kernel(CompressArgs a)
             };
             auto wait_rec = [&]() {
                 owned = true;
-                if (!mbar_wait(bar_rec_free(rs), rpar ^ 1u, s_abort)) dead = true;
+                if (!mbar_wait_warp(bar_rec_free(rs), rpar ^ 1u, s_abort, a.wait_ns)) dead = true;
             };
             if (!done && live)
                 meta = encode_page(in, a.scheme & ~SPECKV_GROUPED, (a.scheme & SPECKV_GROUPED) != 0,
@@ -450,7 +450,7 @@ __global__ void __launch_bounds__(kCThreads, 1) compress_kernel(CompressArgs a)
         bool n_done = false, n_valid = false;
         auto draw = [&]() {
             uint32_t t = lane == 0 ? atomicAdd(&a.scan->ticket, 1u) : 0u;
-            n_tile = __shfl_sync(kFull, t, 0);
+            n_tile = __shfl_sync(kFull, t, 0) + a.ticket0;
             n_done = n_tile >= a.n_tiles;
             n_i = n_tile * kEnc + lane;
             n_sp = 0; n_slot = 0xFFFFFFFFu; n_valid = false;
@@ -467,11 +467,11 @@ __global__ void __launch_bounds__(kCThreads, 1) compress_kernel(CompressArgs a)
             const uint32_t tile = n_tile, i = n_i, sp = n_sp, slot = n_slot;
             const bool done = n_done, valid = n_valid;
             if (!done) draw();
-            if (!mbar_wait(bar_in_empty, (j & 1u) ^ 1u, s_abort)) {                                 // page buffers are free
+            if (!mbar_wait_warp(bar_in_empty, (j & 1u) ^ 1u, s_abort, a.wait_ns)) {                                 // page buffers are free
                 give_up(0xFFFFFFF2u);
                 // giving up: the previous tile's loads may still be in flight towards this CTA's shared
                 // memory; stay (bounded) until they have landed, so that the memory outlives them
-                if (j > 0 && lane < kEnc) mbar_wait(bar_in_full(lane), (j - 1u) & 1u);
+                if (j > 0 && lane < kEnc) mbar_wait(bar_in_full(lane), (j - 1u) & 1u, nullptr, a.wait_ns);
                 return;
             }
             if (lane < kEnc) {
@@ -500,7 +500,7 @@ __global__ void __launch_bounds__(kCThreads, 1) compress_kernel(CompressArgs a)
     bool chain_ok = true;
     for (uint32_t j = 0;; ++j) {
         const uint32_t rs = j % kRecStages, rpar = (j / kRecStages) & 1u;
-        if (!mbar_wait(bar_enc_done(rs), rpar, s_abort)) { give_up(0xFFFFFFF3u); break; }
+        if (!mbar_wait_warp(bar_enc_done(rs), rpar, s_abort, a.wait_ns)) { give_up(0xFFFFFFF3u); break; }
         volatile uint32_t *r = s_ring + (j % kRing) * kRingWords;
         const uint32_t tile = r[0];
         if (tile >= a.n_tiles) break;                                // the loader ran out of tiles
@@ -628,6 +628,6 @@ extern "C" int speckv_compress_static(const void *src, uint32_t n_src_pages, con
     a.src = (const uint4 *)src; a.src_page = src_page; a.dst_slot = dst_slot;
     a.pool = (uint8_t *)pool; a.pte = (unsigned long long *)pte; a.ctl = reinterpret_cast<Ctl *>(ctl); a.scan = su.scan;
     a.pool_gran = pool_bytes / kGranule; a.n_slots = n_slots;
-    a.n_src_pages = n_src_pages; a.n = n; a.n_tiles = n_tiles; a.spin_limit = 4u << 20; a.scheme = scheme;
+    a.n_src_pages = n_src_pages; a.n = n; a.n_tiles = n_tiles; a.spin_limit = kDefaultSpinLimit; a.wait_ns = kDefaultWaitNs; a.ticket0 = 0; a.scheme = scheme;
     return launch_compress(a, su.n_sm, st) == cudaSuccess ? 0 : SPECKV_E_CUDA;
 }

@@ -18,7 +18,9 @@ struct speckv_ctx {
     ScanScratch *scan;
     uint32_t scan_tiles;   // capacity of scan->tile
     uint32_t epoch;        // gather calls so far (prefetch residency filter)
-    uint32_t spin_limit;
+    uint32_t spin_limit;            // look-back polls per window (speckv_set_wait_limits)
+    unsigned long long wait_ns;     // time limit of barrier waits
+    uint32_t missing_tiles;         // fault injection for the next speckv_compress (speckv_inject_missing_tiles)
     // Gather launches still possibly in flight since the last ordinary (fully ordered) launch: their
     // destination ranges, and whether any of them skipped the wait for its predecessor.
     struct Span { uintptr_t lo, hi; };
@@ -90,7 +92,9 @@ int speckv_create(speckv_ctx **out, const speckv_config *cfg)
     c->n_slots = (unsigned long long)cfg->n_layers * cfg->blocks_per_layer * 2ull * cfg->n_kv_heads;
     c->epoch = 0;
     c->n_span = 0; c->chain_live = false; c->chain_skipped = false; c->chain_stream = nullptr;
-    c->spin_limit = 4u << 20;   // polls of >= 64 ns each per look-back window: gives up after a few seconds
+    c->spin_limit = kDefaultSpinLimit;
+    c->wait_ns = kDefaultWaitNs;
+    c->missing_tiles = 0;
     unsigned long long tiles = (c->n_slots + compress_tile_pages() - 1) / compress_tile_pages() + 1;
     c->scan_tiles = (uint32_t)(tiles > 0xFFFFFFFFull ? 0xFFFFFFFFull : tiles);
     bool ok = cudaMalloc(&c->pool, cfg->pool_bytes) == cudaSuccess &&
@@ -132,6 +136,21 @@ int speckv_reset(speckv_ctx *c, void *stream)
     return clear_ctl(c, true, st);
 }
 
+int speckv_set_wait_limits(speckv_ctx *c, uint32_t lookback_polls, uint64_t wait_ns)
+{
+    if (!c) return SPECKV_E_ARG;
+    c->spin_limit = lookback_polls ? lookback_polls : kDefaultSpinLimit;
+    c->wait_ns = wait_ns ? wait_ns : kDefaultWaitNs;
+    return 0;
+}
+
+int speckv_inject_missing_tiles(speckv_ctx *c, uint32_t n_tiles)
+{
+    if (!c) return SPECKV_E_ARG;
+    c->missing_tiles = n_tiles;
+    return 0;
+}
+
 int speckv_clear_status(speckv_ctx *c, void *stream)
 {
     if (!c) return SPECKV_E_ARG;
@@ -163,6 +182,9 @@ int speckv_compress(speckv_ctx *c, const void *src, uint32_t n_src_pages, const 
     a.pool = c->pool; a.pte = c->pte; a.ctl = c->ctl; a.scan = c->scan;
     a.pool_gran = c->cfg.pool_bytes / kGranule; a.n_slots = c->n_slots;
     a.n_src_pages = n_src_pages; a.n = n; a.n_tiles = n_tiles; a.spin_limit = c->spin_limit; a.scheme = scheme;
+    a.wait_ns = c->wait_ns;
+    a.ticket0 = c->missing_tiles;   // one call only
+    c->missing_tiles = 0;
     return launch_compress(a, c->n_sm, st) == cudaSuccess ? 0 : SPECKV_E_CUDA;
 }
 

@@ -102,9 +102,14 @@ struct CompressArgs {
     Ctl *ctl;
     ScanScratch *scan;
     unsigned long long pool_gran, n_slots;
-    uint32_t n_src_pages, n, n_tiles, spin_limit;
+    uint32_t n_src_pages, n, n_tiles;
+    uint32_t spin_limit;            // polls of one look-back window before the scan gives up
+    unsigned long long wait_ns;     // time limit of every wait on a shared-memory barrier
+    uint32_t ticket0;               // first tile number drawn (0 except under fault injection: lower tiles never appear)
     int scheme;
 };
+constexpr uint32_t kDefaultSpinLimit = 4u << 20;               // >= 200 ns per poll: gives up after a few seconds
+constexpr unsigned long long kDefaultWaitNs = 2000000000ull;
 struct GatherArgs {
     const uint8_t *pool;
     const unsigned long long *pte;

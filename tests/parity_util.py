@@ -88,7 +88,9 @@ class Pair:
 
     def compact(self):
         self.cpu.compact()
-        scratch = self.torch.empty(self.gpu.compact_scratch_bytes(), dtype=self.torch.uint8, device=self.dev)
+        # zeroed like the oracle's: when shared records overflow the pool, the granules between the last copy
+        # that fitted and the end of the pool come back from the scratch area as they were
+        scratch = self.torch.zeros(self.gpu.compact_scratch_bytes(), dtype=self.torch.uint8, device=self.dev)
         self.gpu.compact(scratch)
 
     # ---- the consumer: decode-step attention ---------------------------------------------

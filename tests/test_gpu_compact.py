@@ -60,3 +60,38 @@ def test_compaction_over_many_blocks_with_rewrites_raw_pages_and_bad_entries():
         pr.gather(layer, w.block_table, w.seq_lens, w.dst_tok_off())
     pr.check_state()
     pr.close()
+
+
+def test_entries_sharing_records_overflow_the_pool():
+    """Two slots pointing at one record each get a copy of their own; when the copies no longer fit, the
+    excess is reported POOL_FULL, cleared, and still counted by the cursor.  Same case as the oracle's
+    hand-worked pin, then a larger one that crosses 1,024-slot blocks."""
+    pr = Pair(1, 1, 4, 4, 1, 64 * 12)
+    zero, const = np.zeros(2048, np.uint16), np.full(2048, 3.5, np.float16).view(np.uint16)
+    pr.compress(np.stack([zero, const]), [0, 1], [0, 2], 3)
+    for pte in (pr.cpu.pte, pr.gpu.pte_view().view(pr.torch.int64)):
+        pte[1] = int(pr.cpu.pte[0]); pte[3] = int(pr.cpu.pte[2])
+    pr.compact()
+    pr.check_state()
+    st = pr.gpu.status()
+    assert pr.gpu.cursor() == 20 and st["count"][O.ST_POOL_FULL] == 2 and st["first"][O.ST_POOL_FULL] == 2
+    pr.close()
+
+    w = workloads.llama70b(seed=3, n_layers=2, batch=4, seq=448)                   # 1,792 slots per layer, layer 0 written
+    pool_bytes = 64 * 70000
+    pr = Pair.for_workload(w, pool_bytes=pool_bytes)
+    slots = w.layer_slots(0)
+    pr.compress(w.gen_pages(slots), np.arange(len(slots)), slots, 3)
+    used = pr.gpu.cursor()
+    assert used < 70000 < 2 * used                                                 # one copy fits, two do not
+    free = w.layer_slots(1).astype(np.int64)                                       # layer 1's entries share layer 0's records
+    gpte = pr.gpu.pte_view().view(pr.torch.int64)
+    gpte[pr.torch.from_numpy(free).to(pr.dev)] = gpte[pr.torch.from_numpy(slots.astype(np.int64)).to(pr.dev)]
+    pr.cpu.pte[free] = pr.cpu.pte[slots]
+    pr.compact()
+    pr.check_state()
+    st = pr.gpu.status()
+    assert pr.gpu.cursor() == 2 * used and 0 < st["count"][O.ST_POOL_FULL] < len(slots)
+    live = int((pr.cpu.pte >> 56 & 1).sum())
+    assert live == 2 * len(slots) - st["count"][O.ST_POOL_FULL]
+    pr.close()

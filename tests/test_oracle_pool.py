@@ -371,3 +371,73 @@ def test_compaction_reorders_to_slot_order_and_clears_entries_outside_the_pool()
         assert (e & 0xFFFFFFFF) == at and bytes(pool.pool[at * 64:at * 64 + len(recs[s])]) == recs[s]
         at += (len(recs[s]) + 63) // 64
     assert pool.cursor.value == at
+
+
+def test_compaction_with_entries_that_share_records_in_a_pool_too_small_for_the_copies():
+    """Entries may share a record (nothing forbids two slots pointing at one copy); compaction gives every
+    entry a copy of its own, so the kept total can exceed the pool.  Worked by hand: a 12-granule pool, an
+    all-zero page (273 B -> 5 granules) in slot 0 and a constant page (304 B -> 5 granules) in slot 2, then
+    slot 1 shares slot 0's record and slot 3 shares slot 2's.  In slot order: slot 0 -> granules 0-4,
+    slot 1 -> 5-9, slot 2 would need 10-14 > 12: reported, cleared, and the count still advances to 15 (the
+    cursor rule of the compressor); slot 3 likewise at 15-19.  Cursor 20."""
+    pool = O.Pool(1, 1, 4, 4, 1, 64 * 12)
+    zero, const = np.zeros(2048, np.uint16), _h(np.full(2048, 3.5))
+    pool.compress(np.stack([zero, const]), [0, 1], [0, 2], 3)
+    assert pool.cursor.value == 10
+    rec0, rec2 = O.compress_page(zero, 3), O.compress_page(const, 3)
+    assert (len(rec0), len(rec2)) == (273, 304)
+    pool.pte[1], pool.pte[3] = pool.pte[0], pool.pte[2]
+    pool.clear_status()
+    assert pool.compact() == 0
+    valid = 1 << 56
+    assert [int(e) for e in pool.pte[:4]] == [0 | (273 << 32) | (3 << 48) | valid, 5 | (273 << 32) | (3 << 48) | valid, 0, 0]
+    assert not pool.pte[4:].any()
+    assert pool.cursor.value == 20
+    st = pool.status_dict()
+    assert st["count"][O.ST_POOL_FULL] == 2 and st["first"][O.ST_POOL_FULL] == 2
+    assert sum(st["count"]) == 2
+    for at in (0, 5):                                               # both copies complete, with their zero padding
+        assert bytes(pool.pool[at * 64:at * 64 + 320]) == rec0 + bytes(320 - 273)
+    # a pool with room for three copies keeps three, in slot order
+    pool = O.Pool(1, 1, 4, 4, 1, 64 * 15)
+    pool.compress(np.stack([zero, const]), [0, 1], [0, 2], 3)
+    pool.pte[1], pool.pte[3] = pool.pte[0], pool.pte[2]
+    assert pool.compact() == 0
+    assert [int(e) & 0xFFFFFFFF for e in pool.pte[:3]] == [0, 5, 10] and pool.pte[3] == 0 and pool.cursor.value == 20
+    assert bytes(pool.pool[10 * 64:10 * 64 + 320]) == rec2 + bytes(320 - 304)
+    assert pool.status_dict()["first"][O.ST_POOL_FULL] == 3
+
+
+def test_gather_skips_a_sequence_whose_rows_pass_the_destination_capacity():
+    """Three sequences of 3, 2 and 1 blocks; the destination holds 64 token rows, the second sequence is
+    placed at row 48 (48 + 32 > 64).  All 2 blocks x 2 x H pages of that sequence are reported with the index
+    of its first page = the 3*2*H pages of sequence 0, nothing of it is written, the others are delivered."""
+    w = workloads.llama70b(seed=4, n_layers=1, batch=3, seq=48)
+    w.seq_lens = np.array([48, 20, 5], np.uint32)
+    pool = _fill(w)
+    H = w.n_kv_heads
+    tok = np.array([0, 48, 16 + 32], np.uint64)                     # sequence 2 shares rows 48.. with the skipped one
+    dst = np.full(64 * 2 * H * 128, 0xCDCD, np.uint16)
+    l2 = np.zeros(w.batch * 4 * 2 * H * 2048, np.uint16)
+    assert pool.decompress_gather(0, w.block_table, w.seq_lens, tok, None, dst, l2) == 0
+    st = pool.status_dict()
+    assert st["count"][O.ST_BAD_DST] == 2 * 2 * H and st["first"][O.ST_BAD_DST] == 3 * 2 * H
+    assert sum(st["count"]) == 2 * 2 * H and pool.stats.pages_decoded == (3 + 1) * 2 * H
+    rows = dst.reshape(64, 2 * H * 128)
+    for kv in range(2):                                            # sequence 0: rows 0-47 as [K|V][head][48][128]
+        for h in range(H):
+            for n in range(3):
+                slot = ((0 * w.blocks_per_layer + w.block_table[0][n]) * 2 + kv) * H + h
+                el = ((kv * H + h) * 48 + 16 * n) * 128
+                assert np.array_equal(dst[el:el + 2048], _expected_page(w, slot))
+    for kv in range(2):                                            # sequence 2: one block at row 48
+        for h in range(H):
+            slot = ((0 * w.blocks_per_layer + w.block_table[2][0]) * 2 + kv) * H + h
+            el = 48 * 2 * H * 128 + (kv * H + h) * 16 * 128
+            assert np.array_equal(dst[el:el + 2048], _expected_page(w, slot))
+    assert np.all(rows[48 + 16:] == 0xCDCD)                        # nothing of the skipped sequence was written
+    # exactly at capacity is accepted
+    pool.clear_status()
+    dst2 = np.full(80 * 2 * H * 128, 0xCDCD, np.uint16)
+    assert pool.decompress_gather(0, w.block_table, w.seq_lens[:2], np.array([0, 48], np.uint64), None, dst2, l2) == 0
+    assert sum(pool.status_dict()["count"]) == 0 and not np.any(np.all(dst2.reshape(-1, 2048) == 0xCDCD, axis=1))

@@ -4,8 +4,8 @@ Some users of this library run where cudaMalloc is not an option (an inference s
 gave all device memory to its own allocator at start-up, a plug-in that only receives
 buffers).  For them the library has one entry point that takes every buffer from the caller
 and keeps its scan scratch in a fixed array inside the library.  This test drives it through
-the C ABI and requires the same bytes as the context-based speckv_compress: record log, page
-table and cursor bit for bit, on two calls in a row (the second appends behind the first and
+the C ABI and requires the same bytes as the context-based speckv_compress and as the CPU
+oracle: record log, page table, cursor, status block and counters bit for bit, on two calls in a row (the second appends behind the first and
 reuses the fixed scratch, which still holds the first call's contents).
 Collected last on purpose: a failure here must not hide any other test's result."""
 import numpy as np
@@ -23,12 +23,14 @@ def _ctl_block(torch):
 def test_static_entry_point_matches_context_compress_on_two_calls():
     import torch
     from kvgen import workloads
+    from oracle import oracle as O
     from paper_2512_11920_b200 import Context, SpeckvError, compress_static, STATIC_MAX_PAGES
 
     w = workloads.llama70b(seed=9, n_layers=2, batch=4, seq=448)              # 1,792 pages per layer
     dev = torch.device("cuda:0")
     pool_bytes = w.n_slots * 2368
     ref = Context(w.n_layers, w.n_kv_heads, w.blocks_per_layer, w.max_blocks_per_seq, w.batch, pool_bytes)
+    cpu = O.Pool(w.n_layers, w.n_kv_heads, w.blocks_per_layer, w.max_blocks_per_seq, w.batch, pool_bytes)
     pool = torch.zeros(pool_bytes, dtype=torch.uint8, device=dev)
     pte = torch.zeros(w.n_slots, dtype=torch.int64, device=dev)
     ctl = _ctl_block(torch)
@@ -46,6 +48,7 @@ def test_static_entry_point_matches_context_compress_on_two_calls():
         t_order = torch.from_numpy(order.view(np.int32)).to(dev)
         t_dst = torch.from_numpy(dst.view(np.int32)).to(dev)
         ref.compress(t_src, t_order, t_dst, 3)
+        cpu.compress(src, order, dst, 3)
         compress_static(t_src, t_order, t_dst, 3, pool, pte, ctl)
         torch.cuda.synchronize()
         cursor = int(ctl[:8].view(torch.int64).item())
@@ -57,6 +60,15 @@ def test_static_entry_point_matches_context_compress_on_two_calls():
         st, stats = ref.status(), ref.stats()
         assert got[8:40].view(np.uint32).tolist() == st["count"] and got[40:72].view(np.uint32).tolist() == st["first"]
         assert got[72:104].view(np.uint64).tolist() == stats["pages_mode"] and int(got[104:112].view(np.uint64)[0]) == stats["granules"]
+        # and against the oracle directly, not only through the other entry point
+        assert cursor == cpu.cursor.value
+        assert np.array_equal(pte.cpu().numpy().view(np.uint64), cpu.pte), f"page table differs from the oracle's after call {call}"
+        assert np.array_equal(pool[:used].cpu().numpy(), cpu.pool[:used]), f"record log differs from the oracle's after call {call}"
+        want = cpu.status_dict()
+        assert got[8:40].view(np.uint32).tolist() == want["count"] and got[40:72].view(np.uint32).tolist() == want["first"]
+        cs = cpu.stats.as_dict()
+        assert got[72:160].view(np.uint64).tolist() == cs["pages_mode"] + [cs[k] for k in (
+            "granules", "payload_bytes", "n_runs", "nonfinite", "pages_decoded", "pf_issued", "pf_skipped")]
     assert ref.status()["count"][5] == 1                                      # the bad index was reported by both
     # beyond the fixed capacity: refused with a clear error, nothing enqueued
     big = torch.zeros(STATIC_MAX_PAGES + 1, dtype=torch.int32, device=dev)
