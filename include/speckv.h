@@ -164,7 +164,19 @@ int speckv_translate(speckv_ctx *ctx, const int32_t *block_table, const speckv_v
  * distinct.  dst_l2 must hold max_seqs*4*2*H pages; it may be NULL when n_pf = 0.
  * Page indices reported in the status block count demand pages first (sequence, block, kv,
  * head order) and then 2*H per prefetch entry.
- *   seq_lens uint32[B] tokens   dst_tok_off uint64[B] token rows   B <= max_seqs */
+ *   seq_lens uint32[B] tokens   dst_tok_off uint64[B] token rows   B <= max_seqs
+ *
+ * Ordering.  Work enqueued on `stream` after this call finds all pages of this call and of every earlier
+ * call written, as stream order promises.  Consecutive calls on one stream overlap, though: the library
+ * launches a gather so that it may start while the previous gather's last CTAs are still running
+ * (programmatic dependent launch); it then reads its inputs and fetches records at once, and waits for
+ * the previous gather before it writes a page or touches a residency tag — or, when the host has seen that
+ * destinations are disjoint and there is no prefetch list, only before it ends.  Consequence for the caller:
+ * block_table, seq_lens, dst_tok_off and pf of a call that directly follows another gather on the same
+ * stream must not be produced by a kernel or copy enqueued between the two calls.  If they are, make any
+ * other speckv call in between (speckv_clear_status will do: the next gather is then an ordinary launch),
+ * or switch the overlap off for the context with speckv_set_gather_chaining(ctx, 0). */
+int speckv_set_gather_chaining(speckv_ctx *ctx, int enabled); /* default 1; host-side setting */
 int speckv_decompress_gather(speckv_ctx *ctx, uint32_t layer, const int32_t *block_table,
                              const uint32_t *seq_lens, const uint64_t *dst_tok_off, uint32_t B,
                              const speckv_prefetch *pf, uint32_t n_pf, void *dst_demand,

@@ -32,7 +32,7 @@ EXPORTS = ["speckv_create", "speckv_destroy", "speckv_reset", "speckv_compress",
            "speckv_attend_workspace_bytes", "speckv_attend_dense", "speckv_decompress_attend",
            "speckv_compact_scratch_bytes", "speckv_compact", "speckv_prefetch_step", "speckv_get_status", "speckv_get_stats", "speckv_clear_status", "speckv_pool_ptr",
            "speckv_pte_ptr", "speckv_l2_tag_ptr", "speckv_get_cursor", "speckv_version",
-           "speckv_set_wait_limits", "speckv_inject_missing_tiles"]
+           "speckv_set_wait_limits", "speckv_inject_missing_tiles", "speckv_set_gather_chaining"]
 
 
 class SpeckvError(RuntimeError):
@@ -88,6 +88,7 @@ def load_library(path: str = LIB_PATH):
     lib.speckv_clear_status.argtypes = [vp, vp]
     lib.speckv_set_wait_limits.argtypes = [vp, u32, u64]
     lib.speckv_inject_missing_tiles.argtypes = [vp, u32]
+    lib.speckv_set_gather_chaining.argtypes = [vp, i32]
     lib.speckv_get_cursor.argtypes = [vp, C.POINTER(u64), vp]
     for name in ("speckv_pool_ptr", "speckv_pte_ptr", "speckv_l2_tag_ptr"):
         getattr(lib, name).argtypes = [vp]
@@ -289,6 +290,10 @@ class Context:
     def set_wait_limits(self, lookback_polls: int = 0, wait_ns: int = 0):
         """speckv_set_wait_limits: bounds of the compressor's internal waits (0 = default)."""
         _check(self._lib.speckv_set_wait_limits(self._h, lookback_polls, wait_ns), "speckv_set_wait_limits")
+
+    def set_gather_chaining(self, enabled: bool):
+        """speckv_set_gather_chaining: allow consecutive gathers on one stream to overlap (default on)."""
+        _check(self._lib.speckv_set_gather_chaining(self._h, int(bool(enabled))), "speckv_set_gather_chaining")
 
     def inject_missing_tiles(self, n_tiles: int):
         """speckv_inject_missing_tiles: the next compress call never hands out its first n_tiles tiles."""

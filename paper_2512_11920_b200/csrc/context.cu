@@ -27,7 +27,7 @@ struct speckv_ctx {
     static constexpr int kMaxSpans = 256;
     Span span[kMaxSpans];
     int n_span;
-    bool chain_live, chain_skipped;
+    bool chain_live, chain_skipped, chain_enabled;
     cudaStream_t chain_stream;
 };
 
@@ -35,7 +35,7 @@ struct speckv_ctx {
 static uint32_t plan_gather_chain(speckv_ctx *c, cudaStream_t st, speckv_ctx::Span dst, speckv_ctx::Span l2, bool has_pf)
 {
     uint32_t mode = 0;
-    if (c->chain_live && st == c->chain_stream && c->n_span + 2 <= speckv_ctx::kMaxSpans) {
+    if (c->chain_enabled && c->chain_live && st == c->chain_stream && c->n_span + 2 <= speckv_ctx::kMaxSpans) {
         bool disjoint = true;
         for (int i = 0; i < c->n_span; ++i)
             if (dst.lo < c->span[i].hi && c->span[i].lo < dst.hi) disjoint = false;
@@ -91,7 +91,7 @@ int speckv_create(speckv_ctx **out, const speckv_config *cfg)
     c->n_sm = prop.multiProcessorCount;
     c->n_slots = (unsigned long long)cfg->n_layers * cfg->blocks_per_layer * 2ull * cfg->n_kv_heads;
     c->epoch = 0;
-    c->n_span = 0; c->chain_live = false; c->chain_skipped = false; c->chain_stream = nullptr;
+    c->n_span = 0; c->chain_live = false; c->chain_skipped = false; c->chain_stream = nullptr; c->chain_enabled = true;
     c->spin_limit = kDefaultSpinLimit;
     c->wait_ns = kDefaultWaitNs;
     c->missing_tiles = 0;
@@ -141,6 +141,14 @@ int speckv_set_wait_limits(speckv_ctx *c, uint32_t lookback_polls, uint64_t wait
     if (!c) return SPECKV_E_ARG;
     c->spin_limit = lookback_polls ? lookback_polls : kDefaultSpinLimit;
     c->wait_ns = wait_ns ? wait_ns : kDefaultWaitNs;
+    return 0;
+}
+
+int speckv_set_gather_chaining(speckv_ctx *c, int enabled)
+{
+    if (!c) return SPECKV_E_ARG;
+    c->chain_enabled = enabled != 0;
+    c->chain_live = false;
     return 0;
 }
 

@@ -222,6 +222,10 @@ __global__ void __launch_bounds__(kGThreads, 3) gather_kernel(GatherArgs a)
             st_decoded += 1;
         }
     }
+    // A chained launch that was allowed to skip the wait (independent of its predecessor) still may not
+    // end before it: work ordered after this grid must find the predecessor's pages written too.  Waiting
+    // here, after the last store, costs nothing but keeps completion in stream order.
+    if (!waited || a.chain == 2u) asm volatile("griddepcontrol.wait;" ::: "memory");
     // st_decoded is warp-uniform; st_issued and st_skipped are per lane (one prefetch entry each)
 #pragma unroll
     for (int d = 16; d >= 1; d >>= 1) {

@@ -309,6 +309,38 @@ def test_back_to_back_gathers_keep_stream_order():
     pr.close()
 
 
+def test_a_foreign_consumer_after_chained_gathers_sees_every_earlier_gather():
+    """Gather into x, then an independent gather into y (which the library launches without waiting for the
+    first), then a kernel that is not the library's reads x on the same stream with no synchronisation in
+    between.  Stream order promises that x is complete; 200 repetitions, x refilled each time."""
+    import torch
+    w = workloads.llama70b(seed=8, n_layers=2, batch=16, seq=2048)             # 32,768 pages per layer: a long first gather
+    pr = Pair.for_workload(w, pool_bytes=w.n_slots * 2368)
+    for layer in range(2):
+        slots = w.layer_slots(layer)
+        pr.compress(w.gen_pages(slots), np.arange(len(slots)), slots, 3)
+    n = w.demand_tokens() * 2 * w.n_kv_heads * 128
+    small_lens = np.full(w.batch, 16, np.uint32)                                # the second gather is short: it ends first
+    x = torch.empty(n, dtype=torch.int16, device="cuda")
+    y = torch.empty(16 * w.batch * 2 * w.n_kv_heads * 128, dtype=torch.int16, device="cuda")
+    bt, lens, tok = pr.t(w.block_table), pr.t(w.seq_lens), pr.t(w.dst_tok_off())
+    lens2, tok2 = pr.t(small_lens), pr.t(w.dst_tok_off(small_lens))
+    d = np.zeros(n, np.uint16)
+    l2 = np.zeros(w.batch * 4 * 2 * w.n_kv_heads * 2048, np.uint16)
+    pr.cpu.decompress_gather(0, w.block_table, w.seq_lens, w.dst_tok_off(), None, d, l2)
+    want = int(d.view(np.int16).astype(np.int64).sum())
+    sums = torch.zeros(200, dtype=torch.int64, device="cuda")
+    for rep in range(200):
+        x.fill_(1)
+        pr.gpu.clear_status()                                                   # the first gather of a repetition is an ordinary launch
+        pr.gpu.decompress_gather(0, bt, lens, tok, x)
+        pr.gpu.decompress_gather(1, bt, lens2, tok2, y)
+        sums[rep] = x.sum(dtype=torch.int64)
+    got = sums.cpu().numpy()
+    assert np.all(got == want), f"{np.count_nonzero(got != want)} of 200 reductions ran before the first gather had finished"
+    pr.close()
+
+
 def test_gather_warps_walk_several_batches_of_pages_with_faults_and_prefetch():
     """A layer large enough that every warp of the gather delivers more than 32 pages (its translation
     runs lane-parallel in batches of 32): mixed raw and packed records, unmapped blocks, cleared
