@@ -129,7 +129,9 @@ int speckv_reset(speckv_ctx *ctx, void *stream);
  *   src          fp16 pages, 16-byte aligned          src_page, dst_slot   uint32[n]
  *   n_src_pages  number of pages readable at src      scheme  SPECKV_RAW .. SPECKV_AUTO,
  *                                                              optionally | SPECKV_GROUPED
- * n = 0 is a no-op.  Calls on one context must be issued on one stream, or be ordered by
+ * n = 0 is a no-op; n may not exceed the context's number of slots (SPECKV_E_TOO_LARGE: the scan scratch
+ * is sized once, at speckv_create, and the call never allocates or synchronises).
+ * Calls on one context must be issued on one stream, or be ordered by
  * the caller, with these exceptions: reading calls (speckv_decompress_gather, speckv_translate,
  * speckv_attend_dense, speckv_decompress_attend) may run on other streams at the same time as
  * each other — provided their outputs do not overlap and at most one of them carries a prefetch
@@ -161,7 +163,11 @@ int speckv_translate(speckv_ctx *ctx, const int32_t *block_table, const speckv_v
  * (seq, l2_slot) is already tagged with this (layer, block) the entry is skipped, otherwise
  * its 2*H pages are written to dst_l2[seq][l2_slot][kv][head][16][128] and the slot is
  * retagged; a stale slot is simply overwritten.  (seq, l2_slot) pairs in one call must be
- * distinct.  dst_l2 must hold max_seqs*4*2*H pages; it may be NULL when n_pf = 0.
+ * distinct.  The tag names the block, not the bytes: it does not notice that the block's slots were
+ * compressed again since (a tail block that decode keeps filling), nor that dst_l2 is another buffer than
+ * last time.  Pass the same dst_l2 for the life of the tags, and after rewriting a block that may sit in
+ * the buffer clear its tag (speckv_l2_tag_ptr: a zero word = empty) or all tags (speckv_reset) — the lazy
+ * invalidation of Sec. 3.4.3 is the overwrite by the next different block, nothing more.  dst_l2 must hold max_seqs*4*2*H pages; it may be NULL when n_pf = 0.
  * Page indices reported in the status block count demand pages first (sequence, block, kv,
  * head order) and then 2*H per prefetch entry.
  *   seq_lens uint32[B] tokens   dst_tok_off uint64[B] token rows   B <= max_seqs
@@ -314,7 +320,9 @@ int speckv_prefetch_step(speckv_ctx *ctx, uint32_t layer, uint32_t back, const i
  *                     0xFFFFFFFF (cudaMemset calls on its own buffer)
  *   n                 at most SPECKV_STATIC_MAX_PAGES pages per call, else SPECKV_E_TOO_LARGE
  * The first call on a device looks up the address of the fixed array (no allocation) and should
- * therefore be made before any stream capture begins.  All calls on a device share the array: each
+ * therefore be made before any stream capture begins; that look-up is serialised, so first calls from
+ * several host threads are safe.  ctl and pte must be 8-byte aligned, src_page and dst_slot 4-byte
+ * aligned (SPECKV_E_ARG otherwise).  All calls on a device share the array: each
  * call clears the part it uses, and two calls whose kernels could overlap on the GPU (different
  * streams without ordering, several host threads) would corrupt each other's scan — issue them on
  * one stream or order them. */

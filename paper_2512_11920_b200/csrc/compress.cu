@@ -19,6 +19,8 @@
 // measured against 2 CTAs x 8 encoders x 4 stages it is 5 % faster (five encoder warps per
 // scheduler instead of four, two control warps per SM instead of four), and the number of
 // stages matters more than anything else (two stages: -11 %).
+#include <mutex>
+
 #include "async_ptx.cuh"
 #include "speckv_dev.cuh"
 
@@ -586,6 +588,7 @@ static __device__ __align__(256) unsigned long long g_static_scan[2 + kStaticMax
 
 struct StaticSetup { ScanScratch *scan; int n_sm; bool ready; };
 static StaticSetup g_static_setup[64];   // per device ordinal
+static std::mutex g_static_mutex;
 
 }  // namespace speckv
 
@@ -599,25 +602,32 @@ extern "C" int speckv_compress_static(const void *src, uint32_t n_src_pages, con
     if (n > SPECKV_STATIC_MAX_PAGES) return SPECKV_E_TOO_LARGE;
     if (n == 0) return 0;
     if (!src || !src_page || !dst_slot || !pool || !pte || !ctl || ((uintptr_t)src & 15u) || ((uintptr_t)pool & 63u) ||
+        (((uintptr_t)ctl | (uintptr_t)pte) & 7u) || (((uintptr_t)src_page | (uintptr_t)dst_slot) & 3u) ||
         pool_bytes == 0 || pool_bytes % kGranule || pool_bytes / kGranule > 0xFFFFFFFFull || n_slots == 0)
         return SPECKV_E_ARG;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return SPECKV_E_CUDA;
     if (dev < 0 || dev >= 64) return SPECKV_E_ARG;
-    StaticSetup &su = g_static_setup[dev];
-    if (!su.ready) {
+    StaticSetup su;
+    {
         // Once per device, with that device current: in host code the array's name is only a handle,
-        // the address the kernel needs comes from the runtime.
-        int major = 0, n_sm = 0;
-        void *p = nullptr;
-        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            return SPECKV_E_CUDA;
-        if (major != 10) return SPECKV_E_DEVICE;
-        if (cudaGetSymbolAddress(&p, g_static_scan) != cudaSuccess || !p) { cudaGetLastError(); return SPECKV_E_CUDA; }
-        su.scan = reinterpret_cast<ScanScratch *>(p);
-        su.n_sm = n_sm;
-        su.ready = true;
+        // the address the kernel needs comes from the runtime.  Under a lock, so that two host threads
+        // making their first call at the same time both see a complete entry.
+        std::lock_guard<std::mutex> guard(g_static_mutex);
+        StaticSetup &slot = g_static_setup[dev];
+        if (!slot.ready) {
+            int major = 0, n_sm = 0;
+            void *p = nullptr;
+            if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+                cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+                return SPECKV_E_CUDA;
+            if (major != 10) return SPECKV_E_DEVICE;
+            if (cudaGetSymbolAddress(&p, g_static_scan) != cudaSuccess || !p) { cudaGetLastError(); return SPECKV_E_CUDA; }
+            slot.scan = reinterpret_cast<ScanScratch *>(p);
+            slot.n_sm = n_sm;
+            slot.ready = true;
+        }
+        su = slot;
     }
     cudaStream_t st = (cudaStream_t)stream;
     const uint32_t n_tiles = (n + kEnc - 1) / kEnc;

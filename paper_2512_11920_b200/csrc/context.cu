@@ -172,18 +172,12 @@ int speckv_compress(speckv_ctx *c, const void *src, uint32_t n_src_pages, const 
     if (!c || scheme < 0 || (scheme & ~SPECKV_GROUPED) > SPECKV_AUTO) return SPECKV_E_ARG;
     if (n == 0) return 0;
     c->chain_live = false;
-    if (!src || !src_page || !dst_slot || ((uintptr_t)src & 15u)) return SPECKV_E_ARG;
+    if (!src || !src_page || !dst_slot || ((uintptr_t)src & 15u) || (((uintptr_t)src_page | (uintptr_t)dst_slot) & 3u))
+        return SPECKV_E_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     const uint32_t tp = compress_tile_pages();
     const uint32_t n_tiles = (uint32_t)(((unsigned long long)n + tp - 1) / tp);
-    if (n_tiles > c->scan_tiles) {   // grow the scan scratch (rare: a call longer than the page table)
-        if (cudaStreamSynchronize(st) != cudaSuccess) return SPECKV_E_CUDA;
-        ScanScratch *p = nullptr;
-        if (cudaMalloc(&p, scan_bytes(n_tiles)) != cudaSuccess) { cudaGetLastError(); return SPECKV_E_CUDA; }
-        cudaFree(c->scan);
-        c->scan = p;
-        c->scan_tiles = n_tiles;
-    }
+    if (n_tiles > c->scan_tiles) return SPECKV_E_TOO_LARGE;   // more pages in one call than the context has slots
     if (cudaMemsetAsync(c->scan, 0, scan_bytes(n_tiles), st) != cudaSuccess) return SPECKV_E_CUDA;
     CompressArgs a;
     a.src = (const uint4 *)src; a.src_page = src_page; a.dst_slot = dst_slot;
@@ -335,7 +329,7 @@ int speckv_prefetch_step(speckv_ctx *c, uint32_t layer, uint32_t back, const int
     if (B == 0) return 0;
     if (!block_table || !access || !cand || !state || !cnt || !l2 || !miss_dst || !where || ((uintptr_t)l2 & 15u) ||
         ((uintptr_t)miss_dst & 15u) || ((uintptr_t)where & 15u) || ((uintptr_t)access & 15u) || ((uintptr_t)cand & 15u) ||
-        ((uintptr_t)state & 15u))
+        ((uintptr_t)state & 15u) || ((uintptr_t)cnt & 15u) || ((uintptr_t)block_table & 15u))
         return SPECKV_E_ARG;
     c->chain_live = false;   // ordinary launches: later gathers do not chain past them
     PrefetchArgs a;

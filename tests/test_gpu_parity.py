@@ -92,6 +92,26 @@ def test_empty_calls_and_argument_errors():
             pr.gpu.compress(torch.zeros(2048, dtype=torch.float16, device="cuda"), e32, e32, bad_scheme)
     with pytest.raises(SpeckvError):
         pr.gpu.decompress_gather(5, pr.t(np.zeros((2, 4), np.int32)), None, None, None)
+    # host-side checks only, nothing is launched: misaligned index lists, a list longer than the context has slots
+    src = torch.zeros(2048, dtype=torch.float16, device="cuda")
+    lib, two = pr.gpu._lib, torch.zeros(4, dtype=torch.int32, device="cuda")
+    st = torch.cuda.current_stream().cuda_stream
+    assert lib.speckv_compress(pr.gpu._h, src.data_ptr(), 1, two.data_ptr() + 2, two.data_ptr(), 2, 3, st) == -1
+    assert lib.speckv_compress(pr.gpu._h, src.data_ptr(), 1, two.data_ptr(), two.data_ptr() + 1, 2, 3, st) == -1
+    long = torch.zeros(pr.gpu.n_slots + 64, dtype=torch.int32, device="cuda")
+    with pytest.raises(SpeckvError, match="too many pages"):
+        pr.gpu.compress(src, long, long, 3)
+    pool = torch.zeros(64 * 100, dtype=torch.uint8, device="cuda")
+    ctl = torch.zeros(168, dtype=torch.uint8, device="cuda")
+    pte = torch.zeros(17, dtype=torch.int64, device="cuda")
+    args = lambda pte_p, ctl_p, sp=two.data_ptr(), ds=two.data_ptr(): (
+        src.data_ptr(), 1, sp, ds, 2, 3, pool.data_ptr(), pool.numel(), pte_p, 16, ctl_p, st)
+    assert lib.speckv_compress_static(*args(pte.data_ptr(), ctl.data_ptr() + 4)) == -1          # control block at an odd address
+    assert lib.speckv_compress_static(*args(pte.data_ptr() + 4, ctl.data_ptr())) == -1          # page table at an odd address
+    assert lib.speckv_compress_static(*args(pte.data_ptr(), ctl.data_ptr(), sp=two.data_ptr() + 2)) == -1
+    assert lib.speckv_compress_static(*args(pte.data_ptr(), ctl.data_ptr(), ds=two.data_ptr() + 1)) == -1
+    torch.cuda.synchronize()
+    assert pr.gpu.cursor() == 0 and sum(pr.gpu.status()["count"]) == 0
     pr.close()
 
 
