@@ -110,6 +110,23 @@ __device__ __forceinline__ void smem_or(uint32_t addr, uint32_t v)
     asm volatile("red.shared.or.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 
+// Exclusive prefix sum over the lanes of four byte fields at once.  The caller guarantees that no
+// field's sum over any 31 lanes reaches 256.  The shuffle's own "source lane exists" predicate guards
+// the additions.
+__device__ __forceinline__ uint32_t scan_excl_bytes(uint32_t v)
+{
+    uint32_t e;
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b32 t;\n\t"
+                 "shfl.sync.up.b32 %0|p, %1, 1, 0, 0xffffffff;\n\t@!p mov.b32 %0, 0;\n\t"
+                 "shfl.sync.up.b32 t|p, %0, 1, 0, 0xffffffff;\n\t@p add.u32 %0, %0, t;\n\t"
+                 "shfl.sync.up.b32 t|p, %0, 2, 0, 0xffffffff;\n\t@p add.u32 %0, %0, t;\n\t"
+                 "shfl.sync.up.b32 t|p, %0, 4, 0, 0xffffffff;\n\t@p add.u32 %0, %0, t;\n\t"
+                 "shfl.sync.up.b32 t|p, %0, 8, 0, 0xffffffff;\n\t@p add.u32 %0, %0, t;\n\t"
+                 "shfl.sync.up.b32 t|p, %0, 16, 0, 0xffffffff;\n\t@p add.u32 %0, %0, t;\n\t}"
+                 : "=&r"(e) : "r"(v));
+    return e;
+}
+
 // ---------------------------------------------------------------- encoder warp: one page
 
 // Reads the page from `in` (shared memory), builds the record in `rec` (shared memory, filled by
@@ -219,27 +236,21 @@ __device__ __forceinline__ uint4 encode_page(const uint4 *in, int scheme, bool g
             for (int k = 0; k < 8; ++k) pay[k * 32 + lane] = make_uint2(q[k][0], q[k][1]);
         } else {
             mode = SPECKV_INT8_DELTA_RLE;
-            // ---- table lookup per group, then the offset of each group's run values: prefix sum
-            // of popcounts in (k, lane) order
+            // ---- offset of each group's run values: exclusive prefix sum of the popcounts in (k, lane)
+            // order.  Within a group row the exclusive sums stay below 8 * 31 = 248, so four rows share a
+            // word as byte fields and nothing carries between them; the row totals (up to 256) are warp
+            // reductions, and the rows' bases accumulate from them.
             uint32_t c[8];
 #pragma unroll
             for (int k = 0; k < 8; ++k) c[k] = __popc(mk[k]);
-            uint32_t pa = c[0] | (c[1] << 10) | (c[2] << 20);   // 10-bit fields hold sums up to 256
-            uint32_t pb_ = c[3] | (c[4] << 10) | (c[5] << 20);
-            uint32_t pc = c[6] | (c[7] << 10);
-            const uint32_t ca = pa, cb = pb_, cc = pc;
+            uint32_t ea = scan_excl_bytes(c[0] + (c[1] << 8) + (c[2] << 16) + (c[3] << 24));
+            uint32_t eb = scan_excl_bytes(c[4] + (c[5] << 8) + (c[6] << 16) + (c[7] << 24));
+            uint32_t excl[8], tot[8];
 #pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                uint32_t ta = __shfl_up_sync(kFull, pa, d), tb = __shfl_up_sync(kFull, pb_, d),
-                         tc = __shfl_up_sync(kFull, pc, d);
-                if (lane >= (uint32_t)d) { pa += ta; pb_ += tb; pc += tc; }
+            for (int k = 0; k < 8; ++k) {
+                excl[k] = __byte_perm(k < 4 ? ea : eb, 0u, 0x4440 + (k & 3));
+                tot[k] = __reduce_add_sync(kFull, c[k]);
             }
-            const uint32_t ta = __shfl_sync(kFull, pa, 31), tb = __shfl_sync(kFull, pb_, 31), tc = __shfl_sync(kFull, pc, 31);
-            pa -= ca; pb_ -= cb; pc -= cc;          // exclusive within the group row
-            const uint32_t excl[8] = {pa & 1023u, (pa >> 10) & 1023u, pa >> 20, pb_ & 1023u, (pb_ >> 10) & 1023u, pb_ >> 20,
-                                      pc & 1023u, pc >> 10};
-            const uint32_t tot[8] = {ta & 1023u, (ta >> 10) & 1023u, ta >> 20, tb & 1023u, (tb >> 10) & 1023u, tb >> 20,
-                                     tc & 1023u, tc >> 10};
             wait_rec();
             // zero the value area and the padding (values are OR-ed in), store the bitmap
             {
@@ -263,8 +274,8 @@ __device__ __forceinline__ uint4 encode_page(const uint4 *in, int scheme, bool g
                 const uint4 e = lut[mk[k]];
                 const uint32_t lo = __byte_perm(q[k][0], q[k][1], e.x) & e.z;        // PRMT reads 16 selector bits
                 const uint32_t hi = __byte_perm(q[k][0], q[k][1], e.y) & e.w;
-                const uint32_t sh = o << 3;          // shifts use the low 5 bits: 8 * (o & 3)
-                const uint32_t w0 = lo << (sh & 31u), w1 = __funnelshift_l(lo, hi, sh), w2 = __funnelshift_l(hi, 0u, sh);
+                const uint32_t sh = o << 3;          // funnel shifts use the low 5 bits: 8 * (o & 3)
+                const uint32_t w0 = __funnelshift_l(0u, lo, sh), w1 = __funnelshift_l(lo, hi, sh), w2 = __funnelshift_l(hi, 0u, sh);
                 const uint32_t p = vals + (o & ~3u);
                 smem_or(p, w0); smem_or(p + 4, w1);
                 smem_or(p + 8, w2);
