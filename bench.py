@@ -115,7 +115,7 @@ class Bench:
         self.scales = torch.from_numpy(w.scales).to(dev)
         for l in range(w.n_layers):
             gen_device.fill(self.src[l * ppl * 2048:(l + 1) * ppl * 2048], w.seed, l * ppl, ppl, self.scales, ppl, w.n_kv_heads)
-        pool_bytes = ((self.pages * 2368 + (64 << 20)) // 64) * 64
+        pool_bytes = ((self.pages * (4160 if (scheme & 15) == 0 else 2368) + (64 << 20)) // 64) * 64   # largest record per page
         self.ctx = Context(w.n_layers, w.n_kv_heads, w.blocks_per_layer, w.max_blocks_per_seq, w.batch, pool_bytes)
         # compress lists a layer's pages in physical slot order (source and page table share the numbering)
         self.idx_all = torch.arange(self.pages, dtype=torch.int32, device=dev)

@@ -308,8 +308,8 @@ int speckv_prefetch_step(speckv_ctx *ctx, uint32_t layer, uint32_t back, const i
  * region where an allocation would synchronise the device or fragment a carefully sized heap,
  * or in a plug-in that is only ever given buffers.  speckv_create allocates the pool, the page
  * table and the scan scratch; this call allocates nothing and needs no context: the caller
- * passes every buffer, and the scan scratch (a ticket counter and one 8-byte word per 20-page
- * tile) is a fixed array inside the library, about 205 KiB, present on every GPU that loads the
+ * passes every buffer, and the scan scratch (a ticket counter and one 8-byte word per tile of 16 or
+ * 20 pages) is a fixed array inside the library, 256 KiB, present on every GPU that loads the
  * library until the process ends.
  *
  * Same operation, record format, placement rule and status reporting as speckv_compress.
@@ -354,7 +354,7 @@ int speckv_clear_status(speckv_ctx *ctx, void *stream); /* status and counters; 
 int speckv_set_wait_limits(speckv_ctx *ctx, uint32_t lookback_polls, uint64_t wait_ns);
 
 /* Fault injection for tests of those limits, made on the host: the next speckv_compress call (only)
- * never hands out its first n_tiles tiles of 20 pages, as if the CTAs that drew them had stalled.
+ * never hands out its first n_tiles tiles (20 pages each; 16 with SPECKV_RAW), as if the CTAs that drew them had stalled.
  * Every later tile then waits for sizes that are never published, until its limit runs out.  Nothing
  * faults or traps; combine with short limits.  n_tiles = 0 cancels. */
 int speckv_inject_missing_tiles(speckv_ctx *ctx, uint32_t n_tiles);

@@ -578,23 +578,135 @@ __global__ void __launch_bounds__(kCThreads, 1) compress_kernel(CompressArgs a)
     }
 }
 
+// ---------------------------------------------------------------- scheme SPECKV_RAW: the bypass as a copy
+//
+// A call with scheme SPECKV_RAW stores every page as it is (the uncompressed share of the traffic, which
+// the paper's engine lets bypass the pipeline).  Every record has the same size, so a tile's size is
+// known as soon as its list entries have been read, long before its pages arrive: the chained scan runs
+// ahead of the data and a page leaves for the pool the moment it has landed.  No encoder, no record
+// staging: each of kRawWarps warps owns kRawTile page buffers and takes whole tiles of kRawTile pages
+// (ticket order, as above).  Lane l < kRawTile of a warp handles page l of the tile with bulk copies of
+// its own: global -> its buffer (mbarrier), then header | page | zero padding -> pool.
+constexpr int kRawWarps = 3;
+constexpr uint32_t kRawTile = 16;                                         // pages per tile and per warp
+constexpr uint32_t kRawGran = (kHdrBytes + kPageBytes + kGranule - 1u) / kGranule;   // 65 granules per record
+constexpr uint32_t kRawOffConst = kRawWarps * kRawTile * kPageBytes;      // 64 B: raw-record header + 48 zero bytes
+constexpr uint32_t kRawOffBar = kRawOffConst + 64;                        // [kRawWarps][kRawTile] mbarriers
+constexpr uint32_t kRawSmem = kRawOffBar + kRawWarps * kRawTile * 8;
+static_assert(kRawSmem + 1024 <= 233472, "one CTA per SM");
+
+__global__ void __launch_bounds__(kRawWarps * 32, 1) raw_copy_kernel(CompressArgs a)
+{
+    extern __shared__ __align__(128) uint8_t smem[];
+    const uint32_t tid = threadIdx.x, lane = tid & 31u;
+    const uint32_t warp = __shfl_sync(kFull, tid >> 5, 0);
+    if (tid < 4) reinterpret_cast<uint4 *>(smem + kRawOffConst)[tid] =
+        tid == 0 ? make_uint4(0u, kPageBytes | (kVersion << 24), 0u, 0u) : make_uint4(0u, 0u, 0u, 0u);
+    if (tid < kRawWarps * kRawTile) mbar_init(smem_u32(smem + kRawOffBar) + 8u * tid, 1);
+    mbar_init_fence();
+    fence_async_smem();                     // the constants are read by bulk stores
+    __syncthreads();
+
+    const uint32_t my_buf = smem_u32(smem + (warp * kRawTile + lane) * kPageBytes);     // lanes < kRawTile only
+    const uint32_t my_bar = smem_u32(smem + kRawOffBar) + 8u * (warp * kRawTile + lane);
+    const uint32_t hdr = smem_u32(smem + kRawOffConst);
+    unsigned long long st_pages = 0;
+    uint32_t phase = 0;                     // loads this lane has waited for: its barrier's parity
+    bool chain_ok = true, in_flight = false;
+    for (;;) {
+        uint32_t t = lane == 0 ? atomicAdd(&a.scan->ticket, 1u) : 0u;
+        const uint32_t tile = __shfl_sync(kFull, t, 0) + a.ticket0;
+        if (tile >= a.n_tiles) break;
+        const uint32_t i = tile * kRawTile + lane;
+        uint32_t sp = 0, slot = 0;
+        bool valid = false;
+        if (lane < kRawTile && i < a.n) {
+            sp = a.src_page[i];
+            slot = a.dst_slot[i];
+            valid = sp < a.n_src_pages && slot < a.n_slots;
+            if (!valid) raise_status(a.ctl, SPECKV_ST_BAD_INDEX, i);
+        }
+        const uint32_t vmask = __ballot_sync(kFull, valid);
+        const unsigned long long agg = (unsigned long long)__popc(vmask) * kRawGran;
+        // the tile's size is known: publish it before anything else, later tiles' scans depend on it
+        if (lane == 0 && tile != 0u) *reinterpret_cast<volatile unsigned long long *>(&a.scan->tile[tile]) = kFlagAgg | agg;
+        // this lane's buffer is free once its previous record has been read out of shared memory
+        bulk_wait_read();
+        if (!chain_ok) valid = false;                                // nothing of this tile can be placed any more
+        if (valid) {
+            mbar_expect_tx(my_bar, kPageBytes);
+            bulk_g2s(my_buf, a.src + (size_t)sp * (kPageBytes / 16), kPageBytes, my_bar);
+        }
+        in_flight = valid;
+        unsigned long long base = 0;
+        if (chain_ok) {
+            chain_ok = tile_base(a, tile, agg, lane, base);
+            if (!chain_ok && lane == 0) raise_status(a.ctl, SPECKV_ST_TIMEOUT, tile * kRawTile);
+        } else if (lane == 0) {
+            a.scan->tile[tile] = kFlagFail;                          // keep later tiles from waiting
+        }
+        if (chain_ok && lane == 0 && tile == a.n_tiles - 1) a.ctl->cursor64 = base + agg;
+        if (valid) {
+            // the page must have landed before the buffer is read or reused, whatever became of the scan
+            const bool landed = mbar_wait(my_bar, phase & 1u, nullptr, a.wait_ns);
+            in_flight = !landed;
+            if (landed) phase += 1;
+            if (!landed) raise_status(a.ctl, SPECKV_ST_TIMEOUT, i);
+            else if (chain_ok) {
+                const unsigned long long off64 = base + (unsigned long long)__popc(vmask & ((1u << lane) - 1u)) * kRawGran;
+                if (off64 + kRawGran > a.pool_gran) {
+                    raise_status(a.ctl, SPECKV_ST_POOL_FULL, i);
+                } else {
+                    uint8_t *dst = a.pool + off64 * kGranule;
+                    bulk_s2g(dst, hdr, 16);
+                    bulk_s2g(dst + 16, my_buf, kPageBytes);
+                    bulk_s2g(dst + 16 + kPageBytes, hdr + 16, 48);
+                    bulk_commit();
+                    a.pte[slot] = off64 | ((unsigned long long)(kHdrBytes + kPageBytes) << 32) | kPteValid;   // mode 0
+                    st_pages += 1;
+                }
+            }
+        }
+        if (__any_sync(kFull, in_flight)) break;                     // a copy towards this CTA never completed: stop taking tiles
+    }
+    // Leaving: nothing may still be on its way into this CTA's shared memory, and the stores must have
+    // read it.  (A load that did not complete within its limit gets one more bounded wait.)
+    if (in_flight) mbar_wait(my_bar, phase & 1u, nullptr, a.wait_ns);
+    bulk_wait_all();
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) st_pages += __shfl_xor_sync(kFull, st_pages, d);
+    if (lane == 0 && st_pages) {
+        atomicAdd(&a.ctl->stats[kStMode0], st_pages);
+        atomicAdd(&a.ctl->stats[kStGranules], st_pages * kRawGran);
+        atomicAdd(&a.ctl->stats[kStPayload], st_pages * kPageBytes);
+    }
+}
+
 cudaError_t launch_compress(const CompressArgs &a, int n_sm, cudaStream_t stream)
 {
+    uint32_t grid = a.n_tiles < (uint32_t)n_sm ? a.n_tiles : (uint32_t)n_sm;   // one persistent CTA per SM
+    if ((a.scheme & ~SPECKV_GROUPED) == SPECKV_RAW) {
+        cudaError_t e = cudaFuncSetAttribute(raw_copy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRawSmem);
+        if (e != cudaSuccess) return e;
+        raw_copy_kernel<<<grid, kRawWarps * 32, kRawSmem, stream>>>(a);
+        return cudaGetLastError();
+    }
     cudaError_t e = cudaFuncSetAttribute(compress_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCompressSmem);
     if (e != cudaSuccess) return e;
-    uint32_t grid = a.n_tiles < (uint32_t)n_sm ? a.n_tiles : (uint32_t)n_sm;   // one persistent CTA per SM
     compress_kernel<<<grid, kCThreads, kCompressSmem, stream>>>(a);
     return cudaGetLastError();
 }
 
-uint32_t compress_tile_pages() { return kEnc; }
+// pages per tile (= per ticket) for a scheme, and the smallest of them (sizes the scan scratch)
+uint32_t compress_tile_pages(int scheme) { return (scheme & ~SPECKV_GROUPED) == SPECKV_RAW ? kRawTile : (uint32_t)kEnc; }
+uint32_t compress_min_tile_pages() { return kRawTile < (uint32_t)kEnc ? kRawTile : (uint32_t)kEnc; }
 
 // ---------------------------------------------------------------- entry point without allocation
 
-constexpr uint32_t kStaticMaxTiles = (SPECKV_STATIC_MAX_PAGES + kEnc - 1) / kEnc;
+constexpr uint32_t kStaticMaxTiles = (SPECKV_STATIC_MAX_PAGES + kRawTile - 1) / kRawTile;   // the smaller tile decides
 
 // Scan scratch of speckv_compress_static: ticket counter + one status word per tile.  Lives in
-// every GPU context that loads the library (about 205 KiB) until the process exits.
+// every GPU context that loads the library (256 KiB) until the process exits.
 static __device__ __align__(256) unsigned long long g_static_scan[2 + kStaticMaxTiles];
 
 struct StaticSetup { ScanScratch *scan; int n_sm; bool ready; };
@@ -641,7 +753,8 @@ extern "C" int speckv_compress_static(const void *src, uint32_t n_src_pages, con
         su = slot;
     }
     cudaStream_t st = (cudaStream_t)stream;
-    const uint32_t n_tiles = (n + kEnc - 1) / kEnc;
+    const uint32_t tp = compress_tile_pages(scheme);
+    const uint32_t n_tiles = (n + tp - 1) / tp;
     // the array keeps the previous call's tickets and status words: clear what this call will use
     if (cudaMemsetAsync(su.scan, 0, sizeof(ScanScratch) + (size_t)n_tiles * sizeof(unsigned long long), st) != cudaSuccess)
         return SPECKV_E_CUDA;

@@ -95,7 +95,7 @@ int speckv_create(speckv_ctx **out, const speckv_config *cfg)
     c->spin_limit = kDefaultSpinLimit;
     c->wait_ns = kDefaultWaitNs;
     c->missing_tiles = 0;
-    unsigned long long tiles = (c->n_slots + compress_tile_pages() - 1) / compress_tile_pages() + 1;
+    unsigned long long tiles = (c->n_slots + compress_min_tile_pages() - 1) / compress_min_tile_pages() + 1;
     c->scan_tiles = (uint32_t)(tiles > 0xFFFFFFFFull ? 0xFFFFFFFFull : tiles);
     bool ok = cudaMalloc(&c->pool, cfg->pool_bytes) == cudaSuccess &&
               cudaMalloc(&c->pte, c->n_slots * 8) == cudaSuccess &&
@@ -175,7 +175,7 @@ int speckv_compress(speckv_ctx *c, const void *src, uint32_t n_src_pages, const 
     if (!src || !src_page || !dst_slot || ((uintptr_t)src & 15u) || (((uintptr_t)src_page | (uintptr_t)dst_slot) & 3u))
         return SPECKV_E_ARG;
     cudaStream_t st = (cudaStream_t)stream;
-    const uint32_t tp = compress_tile_pages();
+    const uint32_t tp = compress_tile_pages(scheme);
     const uint32_t n_tiles = (uint32_t)(((unsigned long long)n + tp - 1) / tp);
     if (n_tiles > c->scan_tiles) return SPECKV_E_TOO_LARGE;   // more pages in one call than the context has slots
     if (cudaMemsetAsync(c->scan, 0, scan_bytes(n_tiles), st) != cudaSuccess) return SPECKV_E_CUDA;

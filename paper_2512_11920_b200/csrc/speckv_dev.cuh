@@ -176,7 +176,8 @@ cudaError_t launch_compact(uint8_t *pool, unsigned long long pool_bytes, unsigne
                            Ctl *ctl, uint8_t *scratch, int n_sm, cudaStream_t stream);
 cudaError_t launch_gather(const GatherArgs &a, int n_sm, cudaStream_t stream);
 cudaError_t launch_translate(const TranslateArgs &a, cudaStream_t stream);
-uint32_t compress_tile_pages();
+uint32_t compress_tile_pages(int scheme);
+uint32_t compress_min_tile_pages();
 uint32_t gather_max_seqs();
 
 

@@ -19,6 +19,27 @@ pytestmark = pytest.mark.gpu
 TILE = 20   # pages per tile of the compressor
 
 
+def test_raw_scheme_look_back_runs_out_too():
+    """The copy kernel of scheme 0 has the same chained scan (tiles of 16 pages) and two bounded waits of its
+    own (a page landing in shared memory, the scan): tile 0 withheld, four tiles requested."""
+    w = workloads.tiny(seed=0)
+    pr = Pair.for_workload(w, pool_bytes=w.n_slots * 4160)
+    pr.gpu.set_wait_limits(lookback_polls=2000, wait_ns=50_000_000)
+    dt = _timed_out_call(pr, w, 4 * 16, scheme=0)
+    st = pr.gpu.status()
+    assert st["count"][O.ST_TIMEOUT] == 3 and st["first"][O.ST_TIMEOUT] == 16 and sum(st["count"]) == 3
+    assert dt < 1.0
+    _nothing_was_placed(pr)
+    pr.gpu.clear_status()
+    pr.gpu.set_wait_limits()
+    slots = w.layer_slots(0)
+    pr.compress(w.gen_pages(slots), np.arange(len(slots)), slots, 0)
+    pr.check_state()
+    pr.gather(0, w.block_table, w.seq_lens, w.dst_tok_off())
+    pr.check_state()
+    pr.close()
+
+
 def _timed_out_call(pr, w, n_pages, scheme=3):
     """Compress the first n_pages slots of layer 0 on the GPU only, with tile 0 withheld."""
     torch = pr.torch
