@@ -104,49 +104,66 @@ class ClockSampler:
 class Bench:
     """Device-resident state of one replica: source K/V, context, index tensors, destination."""
 
-    def __init__(self, w, dev, scheme=3):
+    def __init__(self, w, dev, scheme=3, layer0=0, n_layers=None):
+        """Layers [layer0, layer0 + n_layers) of workload w (default: all); the context numbers them from 0."""
         import torch
         from kvgen import device as gen_device
         from paper_2512_11920_b200 import Context
         self.torch, self.w, self.dev, self.scheme = torch, w, dev, scheme
+        self.layer0, self.L = layer0, (w.n_layers - layer0 if n_layers is None else n_layers)
         ppl = w.pages_per_layer
-        self.pages = w.n_layers * ppl
+        self.pages = self.L * ppl
         self.src = torch.empty(self.pages * 2048, dtype=torch.int16, device=dev)
         self.scales = torch.from_numpy(w.scales).to(dev)
-        for l in range(w.n_layers):
-            gen_device.fill(self.src[l * ppl * 2048:(l + 1) * ppl * 2048], w.seed, l * ppl, ppl, self.scales, ppl, w.n_kv_heads)
-        pool_bytes = ((self.pages * (4160 if (scheme & 15) == 0 else 2368) + (64 << 20)) // 64) * 64   # largest record per page
-        self.ctx = Context(w.n_layers, w.n_kv_heads, w.blocks_per_layer, w.max_blocks_per_seq, w.batch, pool_bytes)
+        for l in range(self.L):
+            gen_device.fill(self.src[l * ppl * 2048:(l + 1) * ppl * 2048], w.seed, (layer0 + l) * ppl, ppl, self.scales, ppl, w.n_kv_heads)
+        pool_bytes = ((self.pages * 4160 + (64 << 20)) // 64) * 64          # room for every page stored raw
+        self.ctx = Context(self.L, w.n_kv_heads, w.blocks_per_layer, w.max_blocks_per_seq, w.batch, pool_bytes)
         # compress lists a layer's pages in physical slot order (source and page table share the numbering)
         self.idx_all = torch.arange(self.pages, dtype=torch.int32, device=dev)
-        self.idx = [self.idx_all[l * ppl:(l + 1) * ppl] for l in range(w.n_layers)]
+        self.idx = [self.idx_all[l * ppl:(l + 1) * ppl] for l in range(self.L)]
         self.bt = torch.from_numpy(w.block_table).to(dev)
         self.lens = torch.from_numpy(w.seq_lens.view(np.int32)).to(dev)
         self.tok = torch.from_numpy(w.dst_tok_off().view(np.int64)).to(dev)
         self.layer_elems = w.demand_tokens() * 2 * w.n_kv_heads * 128
-        self.dst = torch.empty(w.n_layers * self.layer_elems, dtype=torch.int16, device=dev)
-        self.demand_pages = w.demand_tokens() // 16 * 2 * w.n_kv_heads * w.n_layers
+        self.dst = torch.empty(self.L * self.layer_elems, dtype=torch.int16, device=dev)
+        self.demand_pages = w.demand_tokens() // 16 * 2 * w.n_kv_heads * self.L
+        self.raw_idx = None                 # set by mixed(): the pages that take the bypass
         torch.cuda.synchronize()
+
+    def mixed(self, fraction=0.3, seed=11):
+        """Splits the page list: a seeded `fraction` of the pages is stored raw by a scheme-0 call (the share of
+        the traffic that bypasses the codec, Sec. 3.5.3: alpha ~ 0.3), the rest by the configured scheme."""
+        torch = self.torch
+        g = torch.Generator(device=self.dev).manual_seed(seed)
+        take = torch.rand(self.pages, device=self.dev, generator=g) < fraction
+        self.raw_take = take
+        self.raw_idx = self.idx_all[take].contiguous()
+        self.packed_idx = self.idx_all[~take].contiguous()
 
     def dst_layer(self, l):
         return self.dst[l * self.layer_elems:(l + 1) * self.layer_elems]
 
     def step(self, ev=None):
         """One pass of the hot path; ev = (e0, e1, e2) CUDA events recorded around the two phases."""
-        w, c = self.w, self.ctx
+        c = self.ctx
         c.reset()
         if ev:
             ev[0].record()
-        c.compress(self.src, self.idx_all, self.idx_all, self.scheme)
+        if self.raw_idx is None:
+            c.compress(self.src, self.idx_all, self.idx_all, self.scheme)
+        else:
+            c.compress(self.src, self.packed_idx, self.packed_idx, self.scheme)
+            c.compress(self.src, self.raw_idx, self.raw_idx, 0)
         if ev:
             ev[1].record()
-        for l in range(w.n_layers):
+        for l in range(self.L):
             c.decompress_gather(l, self.bt, self.lens, self.tok, self.dst_layer(l))
         if ev:
             ev[2].record()
 
     def launches_per_step(self):
-        return 1 + self.w.n_layers
+        return (1 if self.raw_idx is None else 2) + self.L
 
     # ---- the consumer: decode-step attention per layer ---------------------------------------
     def consumer(self, n_q_heads: int, reps: int = 3):
@@ -155,7 +172,7 @@ class Bench:
         Sec. 3.4.4: gathers run up to two layers ahead on a second stream, into a ring of three workspaces;
         (fused) attention straight from the compressed pages.  Returns milliseconds per pass over all layers."""
         torch, w, c = self.torch, self.w, self.ctx
-        L, B = w.n_layers, w.batch
+        L, B = self.L, w.batch
         g = torch.Generator(device=self.dev).manual_seed(7)
         q = torch.randn(B, n_q_heads, 128, device=self.dev, generator=g).to(torch.float16)
         out = torch.empty_like(q)
@@ -192,31 +209,24 @@ class Bench:
             for l in range(L):
                 c.decompress_attend(l, self.bt, self.lens, q, out, ws)
 
-        side = torch.cuda.Stream(device=self.dev)
-        main = torch.cuda.current_stream()
+        # the multi-layer pipelined prefetch is the library's own call: gathers two layers ahead on the context's
+        # fetch stream into the ring of three workspaces, attention on this stream
+        ring_t = self.dst[:R * self.layer_elems]
+        q_all = q.unsqueeze(0).expand(L, B, n_q_heads, 128).contiguous()
+        out_all = torch.empty_like(q_all)
 
         def pipelined():
-            gathered = [torch.cuda.Event() for _ in range(L)]
-            attended = [torch.cuda.Event() for _ in range(L)]
-            start = torch.cuda.Event()
-            start.record(main)
-            side.wait_event(start)
-            for l in range(L):
-                if l >= R:
-                    side.wait_event(attended[l - R])            # the ring slot is free again
-                with torch.cuda.stream(side):
-                    c.decompress_gather(l, self.bt, self.lens, self.tok, ring[l % R])
-                    gathered[l].record(side)
-                main.wait_event(gathered[l])
-                c.attend_dense(ring[l % R], self.lens, self.tok, q, out, ws)
-                attended[l].record(main)
+            c.pipeline_attend(0, L, self.bt, self.lens, self.tok, ring_t, R, q_all, out_all, ws)
 
         res = {"n_q_heads": n_q_heads, "layers": L,
                "gather_ms": timed(gather_only), "attend_dense_ms": timed(attend_only), "serial_ms": timed(serial),
                "pipelined_ms": timed(pipelined), "fused_ms": timed(fused)}
         kv_bytes = self.demand_pages * PAGE
         t_layer, t_pref = res["attend_dense_ms"] / L, res["gather_ms"] / L
-        res["t_effective_model_ms"] = res["attend_dense_ms"] + max(t_pref - 2 * t_layer, 0.0)
+        # Sec. 3.4.4: T_effective = T_compute + max(T_prefetch - 2 T_layer, 0) per layer, with the two stages measured
+        # alone; the paper's fetch engine is a device of its own, here both stages share one GPU's HBM and SMs
+        res["t_effective_model_ms"] = res["attend_dense_ms"] + L * max(t_pref - 2 * t_layer, 0.0)
+        res["t_effective_measured_ms"] = res["pipelined_ms"]
         res["kv_gbs"] = {k[:-3]: kv_bytes / (res[k] * 1e-3) / 1e9 for k in ("attend_dense_ms", "serial_ms", "pipelined_ms", "fused_ms")}
         return res
 
@@ -245,55 +255,79 @@ class Bench:
                 "live_gbs": after * 64 / (t * 1e-3) / 1e9, "status_counts": c.status()["count"]}
 
     # ---- end to end through the host-buffer entry points --------------------------------
-    def e2e(self, steps: int, ring: int = 4):
-        """The same step through the host-buffer entry points: every layer's pages come from pinned host memory
-        and every layer's gathered K/V goes back to pinned host memory.  Uploads + compression run on one
-        stream, gathers + downloads on a second one that follows layer by layer (an event per layer), so the
-        two directions of the host link are busy at the same time."""
+    def e2e(self, steps: int = 3, warmup: int = 1):
+        """The same step through the host-buffer entry points: every layer's own pages come from pinned host
+        memory (a host copy of the whole cache) and every layer's gathered K/V goes back to pinned host memory
+        of its own.  Uploads + compression run on one stream, gathers + downloads on a second one that follows
+        layer by layer (an event per layer), so the two directions of the host link are busy at the same time.
+        If the host cannot pin two copies of the cache, a ring of four layers is recycled instead (said in the
+        result).  Afterwards every layer's host copy is compared with what the device holds."""
         torch, w, c = self.torch, self.w, self.ctx
-        ppl = w.pages_per_layer
-        ring = min(ring, w.n_layers)
-        h_in = torch.empty(ring * ppl * 2048, dtype=torch.int16).pin_memory()
-        h_out = torch.empty(ring * self.layer_elems, dtype=torch.int16).pin_memory()
+        ppl, L = w.pages_per_layer, self.L
+        ring = L
+        try:
+            h_in = torch.empty(L * ppl * 2048, dtype=torch.int16, pin_memory=True)
+            h_out = torch.empty(L * self.layer_elems, dtype=torch.int16, pin_memory=True)
+        except RuntimeError:
+            ring = min(4, L)
+            h_in = torch.empty(ring * ppl * 2048, dtype=torch.int16, pin_memory=True)
+            h_out = torch.empty(ring * self.layer_elems, dtype=torch.int16, pin_memory=True)
         h_in.copy_(self.src[:ring * ppl * 2048])
-        staging = torch.empty(ring * ppl * 2048, dtype=torch.int16, device=self.dev)
+        n_stage = min(4, L)
+        staging = torch.empty(n_stage * ppl * 2048, dtype=torch.int16, device=self.dev)
         local = torch.arange(ppl, dtype=torch.int32, device=self.dev)
         up, down = torch.cuda.Stream(device=self.dev), torch.cuda.Stream(device=self.dev)
         main = torch.cuda.current_stream()
+
+        def one_step():
+            with torch.cuda.stream(up):
+                up.wait_stream(down)                     # the previous step's gathers are done with the pool
+                c.reset()
+            for l in range(L):
+                r, g = l % ring, l % n_stage
+                with torch.cuda.stream(up):
+                    c.compress_host(h_in[r * ppl * 2048:(r + 1) * ppl * 2048], staging[g * ppl * 2048:(g + 1) * ppl * 2048],
+                                    local, self.idx[l], self.scheme)
+                    done = torch.cuda.Event()
+                    done.record(up)
+                with torch.cuda.stream(down):
+                    down.wait_event(done)
+                    c.decompress_gather_host(l, self.bt, self.lens, self.tok, self.dst_layer(l),
+                                             h_out[r * self.layer_elems:(r + 1) * self.layer_elems])
+
+        torch.cuda.synchronize()
+        up.wait_stream(main)
+        down.wait_stream(main)
+        for _ in range(warmup):
+            one_step()
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(main)
         up.wait_event(e0)
         down.wait_event(e0)
         for _ in range(steps):
-            with torch.cuda.stream(up):
-                up.wait_stream(down)                     # the previous step's gathers are done with the pool
-                c.reset()
-            done = [torch.cuda.Event() for _ in range(w.n_layers)]
-            for l in range(w.n_layers):
-                r = l % ring
-                with torch.cuda.stream(up):
-                    c.compress_host(h_in[r * ppl * 2048:(r + 1) * ppl * 2048], staging[r * ppl * 2048:(r + 1) * ppl * 2048],
-                                    local, self.idx[l], self.scheme)
-                    done[l].record(up)
-                with torch.cuda.stream(down):
-                    down.wait_event(done[l])
-                    c.decompress_gather_host(l, self.bt, self.lens, self.tok, self.dst_layer(l),
-                                             h_out[r * self.layer_elems:(r + 1) * self.layer_elems])
+            one_step()
         main.wait_stream(up)
         main.wait_stream(down)
         e1.record(main)
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / steps
-        h2d = w.n_layers * ppl * PAGE
-        d2h = w.n_layers * self.layer_elems * 2
-        # what came back for the last layers is what the device holds, and every page went both ways
+        h2d = L * ppl * PAGE
+        d2h = L * self.layer_elems * 2
+        # every page went both ways, and what came back is what the device holds: layer by layer (the last
+        # `ring` layers when a ring was recycled), compared on the device after an upload of the host copy
         stats, status = c.stats(), c.status()
-        last = w.n_layers - 1
-        same = bool((h_out[(last % ring) * self.layer_elems:(last % ring + 1) * self.layer_elems] == self.dst_layer(last).cpu()).all())
+        checked, same = 0, True
+        for l in range(L - ring, L):
+            r = l % ring
+            back = h_out[r * self.layer_elems:(r + 1) * self.layer_elems].to(self.dev, non_blocking=True)
+            same = same and bool(torch.equal(back, self.dst_layer(l)))
+            checked += 1
         if not same or sum(status["count"]) or sum(stats["pages_mode"]) != self.pages or stats["pages_decoded"] != self.demand_pages:
-            raise RuntimeError(f"end-to-end step inconsistent: {stats} {status} host copy equal: {same}")
-        return ms, h2d, d2h
+            raise RuntimeError(f"end-to-end step inconsistent: {stats} {status} host copies equal: {same}")
+        return {"ms_per_step": ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": steps, "warmup": warmup,
+                "host_buffers": "one pinned copy of the whole cache each way" if ring == L else f"a ring of {ring} layers, recycled",
+                "layers_compared_with_device": checked}
 
     # ---- sampled parity at the benchmarked size -------------------------------------------
     def sampled_parity(self, n_samples: int = 48, seed: int = 123):
@@ -306,11 +340,12 @@ class Bench:
         pool = self.ctx.pool_view()
         bad = 0
         for _ in range(n_samples):
-            l = int(rng.integers(w.n_layers)); b = int(rng.integers(w.batch))
+            l = int(rng.integers(self.L)); b = int(rng.integers(w.batch))
             n = int(rng.integers((int(w.seq_lens[b]) + 15) // 16)); kv = int(rng.integers(2)); h = int(rng.integers(H))
             slot = ((l * w.blocks_per_layer + int(w.block_table[b][n])) * 2 + kv) * H + h
-            page = w.gen_pages([slot])[0]
-            rec = O.compress_page(page, self.scheme)
+            page = w.gen_pages([self.layer0 * ppl + slot])[0]
+            scheme = 0 if self.raw_idx is not None and bool(self.raw_take[slot].item()) else self.scheme
+            rec = O.compress_page(page, scheme)
             e = int(pte[slot].item()) & 0xFFFFFFFFFFFFFFFF
             off, rec_len, mode, valid = (e & 0xFFFFFFFF) * 64, (e >> 32) & 0xFFFF, (e >> 48) & 0xFF, (e >> 56) & 1
             got_rec = pool[off:off + ((len(rec) + 63) // 64) * 64].cpu().numpy().tobytes()
@@ -574,15 +609,119 @@ def run_reference(args, w):
             "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
 
 
+def timed_passes(b, passes: int, warmup: int = 3, sample_clocks: int = -1):
+    """Runs `warmup` untimed and `passes` timed passes of b.step(); returns per-phase mean milliseconds, the
+    total, the context's counters after the last pass and (if sample_clocks >= 0) the clocks seen meanwhile."""
+    import torch
+    for _ in range(warmup):
+        b.step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(sample_clocks) if sample_clocks >= 0 else None
+    if sampler:
+        sampler.start()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(passes)]
+    end = torch.cuda.Event(enable_timing=True)
+    for e in evs:
+        b.step(e)
+    end.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if sampler else None
+    return {"comp_ms": float(np.mean([e[0].elapsed_time(e[1]) for e in evs])),
+            "gath_ms": float(np.mean([e[1].elapsed_time(e[2]) for e in evs])),
+            "total_ms": evs[0][0].elapsed_time(end), "stats": b.ctx.stats(), "status": b.ctx.status(), "clocks": clocks}
+
+
+def phase_figures(b, comp_ms, gath_ms, stats, peak, clocks=None):
+    """GB/s of uncompressed K/V and of algorithmic HBM traffic per phase.  Algorithmic bytes: compress reads the
+    page, its two list entries, and writes the record's granules and one page-table entry; decompress+gather
+    reads the granules, the entry and its share of the block-table entry, and writes the page."""
+    H = b.w.n_kv_heads
+    gran = stats["granules"]                                    # counters were reset at the start of the last pass
+    comp_bytes = b.pages * (PAGE + 8 + 8) + 64 * gran
+    gath_bytes = 64 * gran * (b.demand_pages / b.pages) + b.demand_pages * (8 + 4.0 / (2 * H) + PAGE)
+    out = {}
+    for name, ms, nbytes, pages in (("speckv_compress", comp_ms, comp_bytes, b.pages),
+                                    ("speckv_decompress_gather", gath_ms, gath_bytes, b.demand_pages)):
+        hbm = nbytes / (ms * 1e-3) / 1e9
+        out[name] = {"ms_per_pass": ms, "uncompressed_gbs": pages * PAGE / (ms * 1e-3) / 1e9, "hbm_gbs": hbm,
+                     "hbm_frac_of_measured": hbm / peak, "hbm_frac_of_8000": hbm / 8000.0, "algorithmic_bytes": nbytes}
+        if clocks and clocks.get("sm_mhz"):
+            # time x clock per page: compares runs whose power-capped clocks differ
+            out[name]["gpu_cycles_per_page"] = ms * 1e-3 * clocks["sm_mhz"] * 1e6 / pages
+    return out
+
+
+def free_cuda(*objs):
+    import gc
+    import torch
+    for o in objs:
+        if hasattr(o, "ctx"):
+            o.ctx.close()
+    del objs
+    gc.collect()
+    torch.cuda.empty_cache()
+
+
+def other_workloads(args, dev, peak):
+    """Summary figures of the other configurations: 7B-shaped (whole cache resident), 13B-shaped (50 GiB,
+    streamed in groups of eight layers: generate, compress, fetch back, next group), the decode-step paged
+    fetch and the managed prefetch buffer.  Each with the clocks seen while it was timed."""
+    import torch
+    res = {}
+    w = workloads.llama7b(seed=0)
+    b = Bench(w, dev, args.scheme)
+    t = timed_passes(b, passes=12, warmup=3, sample_clocks=dev.index or 0)
+    res["llama2-7b"] = {"pages": b.pages, "kernels": phase_figures(b, t["comp_ms"], t["gath_ms"], t["stats"], peak, t["clocks"]),
+                        "clocks": t["clocks"], "status_counts": t["status"]["count"], "parity": b.sampled_parity(n_samples=8, seed=7)}
+    free_cuda(b)
+    del b
+    w = workloads.llama13b(seed=0)
+    group, comp_ms, gath_ms, pages, dpages, gran, counts, bad = 8, 0.0, 0.0, 0, 0, 0, np.zeros(8, np.int64), 0
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    for l0 in range(0, w.n_layers, group):
+        b = Bench(w, dev, args.scheme, layer0=l0, n_layers=min(group, w.n_layers - l0))
+        t = timed_passes(b, passes=3, warmup=1)
+        comp_ms += t["comp_ms"]; gath_ms += t["gath_ms"]; pages += b.pages; dpages += b.demand_pages
+        gran += t["stats"]["granules"]; counts += np.array(t["status"]["count"])
+        bad += b.sampled_parity(n_samples=2, seed=l0)["mismatches"]
+        free_cuda(b)
+        del b
+    clocks = sampler.stop()
+    H = w.n_kv_heads
+    cb, gb = pages * (PAGE + 16) + 64 * gran, 64 * gran * (dpages / pages) + dpages * (8 + 4.0 / (2 * H) + PAGE)
+    res["llama2-13b"] = {"pages": pages, "streamed": f"{w.n_layers // group} groups of {group} layers, times summed over the groups",
+                         "kernels": {"speckv_compress": {"ms_per_pass": comp_ms, "uncompressed_gbs": pages * PAGE / comp_ms / 1e6,
+                                                         "hbm_gbs": cb / comp_ms / 1e6, "hbm_frac_of_measured": cb / comp_ms / 1e6 / peak},
+                                     "speckv_decompress_gather": {"ms_per_pass": gath_ms, "uncompressed_gbs": dpages * PAGE / gath_ms / 1e6,
+                                                                  "hbm_gbs": gb / gath_ms / 1e6, "hbm_frac_of_measured": gb / gath_ms / 1e6 / peak}},
+                         "clocks": clocks, "status_counts": [int(x) for x in counts], "parity": {"pages_checked": 2 * (w.n_layers // group), "mismatches": bad}}
+    sub = argparse.Namespace(**vars(args))
+    sub.steps, sub.warmup = 30, 3
+    d = run_decode_fetch(sub, workloads.decode_fetch(seed=0), dev)
+    res["decode-fetch-7b"] = {"uncompressed_gbs": d["value"], "ms_per_step": d["ms_per_step"], "per_step_demand_gbs": d["per_step_demand_gbs"],
+                              "steps_timed": d["steps"], "prefetch": d["prefetch"], "clocks": d["clocks"], "status_counts": d["status_counts"]}
+    torch.cuda.empty_cache()
+    d = run_managed_prefetch(sub, workloads.decode_fetch(seed=0, n_layers=4), dev)
+    res["managed-prefetch-7b"] = {"uncompressed_gbs": d["value"], "us_per_call": d["ms_per_step"] * 1e3, "calls_timed": d["steps"],
+                                  "hit_rate": d["prefetch"]["hit_rate"], "coverage": d["prefetch"]["coverage"],
+                                  "precision": d["prefetch"]["precision"], "clocks": d["clocks"], "status_counts": d["status_counts"]}
+    torch.cuda.empty_cache()
+    return res
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="speckv", choices=["speckv", "reference"])
-    ap.add_argument("--workload", default="llama2-70b-gqa", choices=["llama2-70b-gqa", "llama2-7b", "decode-fetch-7b", "managed-prefetch-7b"])
+    ap.add_argument("--workload", default="llama2-70b-gqa", choices=["llama2-70b-gqa", "llama2-7b", "llama2-13b", "decode-fetch-7b", "managed-prefetch-7b"])
     ap.add_argument("--layers", type=int, default=0, help="use only this many layers (small cases for profiling)")
     ap.add_argument("--scheme", type=int, default=3)
+    ap.add_argument("--passes-per-step", type=int, default=0, help="passes of the hot path per step (0 = enough for --min-seconds)")
+    ap.add_argument("--min-seconds", type=float, default=2.2, help="shortest timed region the automatic passes-per-step aims at")
+    ap.add_argument("--no-workloads", action="store_true", help="skip the summary figures of the other configurations")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-adaptive", action="store_true", help="skip the extra runs with the adaptive and grouped schemes")
@@ -630,7 +769,23 @@ def main():
         return
 
     b = Bench(w, dev, args.scheme)
-    for _ in range(max(args.warmup, 3)):
+    # A step is `passes_per_step` passes of the whole hot path (every layer compressed, every layer fetched
+    # back), chosen from a first measurement so that the timed region covers at least two seconds: shorter
+    # regions end before the power limit has settled the clock.
+    b.step()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(2):
+        b.step()
+    torch.cuda.synchronize()
+    est_ms = (time.perf_counter() - t0) * 1e3 / 2
+    pps = args.passes_per_step or max(1, int(np.ceil(args.min_seconds * 1e3 / (args.steps * est_ms))))
+    if world > 1:                                             # every rank must run the same number of passes
+        t = torch.tensor([pps], dtype=torch.int64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        pps = int(t.item())
+    warm = max(args.warmup, 3)
+    for _ in range(warm * pps):
         b.step()
     torch.cuda.synchronize()
     if world > 1:
@@ -638,11 +793,12 @@ def main():
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    n_pass = args.steps * pps
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n_pass)]
     end = torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
-    for s in range(args.steps):
-        b.step(evs[s])
+    for e in evs:
+        b.step(e)
     end.record()
     torch.cuda.synchronize()
     clocks = sampler.stop() if rank == 0 else None
@@ -660,37 +816,29 @@ def main():
             dist.destroy_process_group()
         return
 
-    # ---- algorithmic bytes (per layer launch) ----------------------------------------------
-    L, H = w.n_layers, w.n_kv_heads
-    ppl, dpl = w.pages_per_layer, b.demand_pages // L
-    gran_layer = stats["granules"] / L                       # counters were reset at the start of the last step
-    comp_bytes = ppl * (PAGE + 8 + 8) + 64 * gran_layer
-    gath_bytes = 64 * gran_layer * (dpl / ppl) + dpl * (8 + 4.0 / (2 * H) + PAGE)
+    L, H = b.L, w.n_kv_heads
     peak, peak_kind = measured_peak_gbs()
-    comp_gbs_unc = b.pages * PAGE / (comp_ms * 1e-3) / 1e9
-    gath_gbs_unc = b.demand_pages * PAGE / (gath_ms * 1e-3) / 1e9
-    comp_hbm = comp_bytes * L / (comp_ms * 1e-3) / 1e9
-    gath_hbm = gath_bytes * L / (gath_ms * 1e-3) / 1e9
+    kern = phase_figures(b, comp_ms, gath_ms, stats, peak, clocks)
     dom = "speckv_compress" if comp_ms >= gath_ms else "speckv_decompress_gather"
-    dom_hbm = comp_hbm if comp_ms >= gath_ms else gath_hbm
-    dom_pages = b.pages if comp_ms >= gath_ms else dpl          # pages per launch of the dominant kernel
-    value = whole_job_gbs((b.pages + b.demand_pages) * PAGE, world, ms_per_step)
+    # the compressor is one launch per pass, the gather one launch per layer
+    dom_pages = b.pages if dom == "speckv_compress" else b.demand_pages // L
+    dom_bytes = kern[dom]["algorithmic_bytes"] / (1 if dom == "speckv_compress" else L)
+    value = whole_job_gbs((b.pages + b.demand_pages) * PAGE * pps, world, ms_per_step)
 
-    out = {"metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+    out = {"metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": warm,
            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16->i8",
            "data": "synthetic",
            "config": {"workload": w.name, "layers": L, "kv_heads": H, "batch": w.batch, "seq": int(w.seq_lens.max()),
                       "pages": b.pages, "uncompressed_gib": b.pages * PAGE / 2 ** 30, "scheme": args.scheme,
+                      "passes_per_step": pps, "timed_seconds": total_ms * 1e-3,
+                      "step": f"{pps} passes of the whole hot path (one compress call over the cache + one gather call per layer each); "
+                              "the repeat makes the timed region long enough for the power-capped clock to settle",
                       "block_table": "seeded random permutation", "l2": "inputs larger than L2 (no flush)",
-                      "parallelism": "replicas only" if world > 1 else "1 GPU", "calls_per_step": b.launches_per_step()},
-           "gpu_launches": b.launches_per_step() * args.steps, "clocks": clocks,
-           "kernels": {"speckv_compress": {"ms_per_step": comp_ms, "uncompressed_gbs": comp_gbs_unc, "hbm_gbs": comp_hbm,
-                                           "hbm_frac_of_measured": comp_hbm / peak, "hbm_frac_of_8000": comp_hbm / 8000.0},
-                       "speckv_decompress_gather": {"ms_per_step": gath_ms, "uncompressed_gbs": gath_gbs_unc, "hbm_gbs": gath_hbm,
-                                                    "hbm_frac_of_measured": gath_hbm / peak, "hbm_frac_of_8000": gath_hbm / 8000.0}},
-           "roofline": {"bound": "hbm", "kernel": dom, "achieved": dom_hbm, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
-                        "frac": dom_hbm / peak, "traffic": ncu_traffic(dom, dom_pages),
-                        "algorithmic_bytes_per_launch": (comp_bytes * L) if comp_ms >= gath_ms else gath_bytes},
+                      "parallelism": "replicas only" if world > 1 else "1 GPU", "calls_per_step": b.launches_per_step() * pps},
+           "gpu_launches": b.launches_per_step() * n_pass, "clocks": clocks, "kernels": kern,
+           "roofline": {"bound": "hbm", "kernel": dom, "achieved": kern[dom]["hbm_gbs"], "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                        "frac": kern[dom]["hbm_gbs"] / peak, "traffic": ncu_traffic(dom, dom_pages),
+                        "algorithmic_bytes_per_launch": dom_bytes},
            "compression": {"stored_ratio": b.pages * PAGE / (64.0 * stats["granules"]) if stats["granules"] else None,
                            "pages_mode": stats["pages_mode"], "status_counts": status["count"]}}
     # The same step with other schemes, reported beside the headline (which keeps every stage of the
@@ -701,19 +849,33 @@ def main():
     if args.scheme == 3 and not args.no_adaptive:
         extras = {"int8_only": 1, "int8_delta": 2,             # the other rows of the paper's compression ablation
                   "adaptive_scheme": 4, "grouped_scales": 3 | 16, "grouped_scales_adaptive": 4 | 16}
+    if extras:
+        extras["raw_only"] = 0                                 # the bypass of Sec. 3.5.3 for every page: a copy
     for name, scheme in extras.items():
         b.scheme = scheme
-        for _ in range(3):
-            b.step()
-        evx = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(5)]
-        for e in evx:
-            b.step(e)
-        torch.cuda.synchronize()
-        cx = float(np.mean([e[0].elapsed_time(e[1]) for e in evx])); gx = float(np.mean([e[1].elapsed_time(e[2]) for e in evx]))
-        stx = b.ctx.stats()
-        out[name] = {"scheme": scheme, "compress_uncompressed_gbs": b.pages * PAGE / (cx * 1e-3) / 1e9,
-                     "gather_uncompressed_gbs": b.demand_pages * PAGE / (gx * 1e-3) / 1e9,
-                     "stored_ratio": b.pages * PAGE / (64.0 * stx["granules"]), "pages_mode": stx["pages_mode"]}
+        t = timed_passes(b, passes=8, warmup=3)
+        k = phase_figures(b, t["comp_ms"], t["gath_ms"], t["stats"], peak)
+        out[name] = {"scheme": scheme, "compress_uncompressed_gbs": k["speckv_compress"]["uncompressed_gbs"],
+                     "gather_uncompressed_gbs": k["speckv_decompress_gather"]["uncompressed_gbs"],
+                     "compress_hbm_frac_of_measured": k["speckv_compress"]["hbm_frac_of_measured"],
+                     "gather_hbm_frac_of_measured": k["speckv_decompress_gather"]["hbm_frac_of_measured"],
+                     "stored_ratio": b.pages * PAGE / (64.0 * t["stats"]["granules"]), "pages_mode": t["stats"]["pages_mode"]}
+    b.scheme = args.scheme
+    if extras:
+        # mixed traffic: a seeded 30 % of the pages take the bypass (a scheme-0 call over them), the rest the codec
+        b.mixed(0.3)
+        t = timed_passes(b, passes=20, warmup=3, sample_clocks=local)
+        k = phase_figures(b, t["comp_ms"], t["gath_ms"], t["stats"], peak, t["clocks"])
+        out["mixed_raw30"] = {"raw_fraction": float(b.raw_idx.numel()) / b.pages, "calls_per_pass": b.launches_per_step(),
+                              "kernels": k, "clocks": t["clocks"], "pages_mode": t["stats"]["pages_mode"],
+                              "stored_ratio": b.pages * PAGE / (64.0 * t["stats"]["granules"]), "status_counts": t["status"]["count"],
+                              "vs_headline": {"compress_uncompressed": k["speckv_compress"]["uncompressed_gbs"] / kern["speckv_compress"]["uncompressed_gbs"],
+                                              "gather_uncompressed": k["speckv_decompress_gather"]["uncompressed_gbs"] / kern["speckv_decompress_gather"]["uncompressed_gbs"],
+                                              "compress_hbm": k["speckv_compress"]["hbm_gbs"] / kern["speckv_compress"]["hbm_gbs"],
+                                              "gather_hbm": k["speckv_decompress_gather"]["hbm_gbs"] / kern["speckv_decompress_gather"]["hbm_gbs"]}}
+        if world == 1 and not args.no_cpu_baseline:
+            out["mixed_raw30"]["parity"] = b.sampled_parity(n_samples=24, seed=9)
+        b.raw_idx = None
     b.scheme = args.scheme
     if args.consumer:
         b.step()
@@ -722,9 +884,8 @@ def main():
     if args.consumer:
         out["lifecycle"] = b.lifecycle()
     if not args.no_e2e:
-        ms, h2d, d2h = b.e2e(steps=1)
-        out["e2e"] = {"value": (b.pages + b.demand_pages) * PAGE / (ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": ms,
-                      "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+        e = b.e2e(steps=3, warmup=1)
+        out["e2e"] = {"value": (b.pages + b.demand_pages) * PAGE / (e["ms_per_step"] * 1e-3) / 1e9, "unit": "GB/s", **e}
     if world == 1 and not args.no_cpu_baseline:
         # the oracle leg: sampled parity of what the timed configuration wrote (and of the extra schemes),
         # then the oracle timed on a bounded sample
@@ -737,7 +898,7 @@ def main():
             torch.cuda.synchronize()
             out[name]["parity"] = b.sampled_parity(n_samples=16, seed=5)
         b.scheme = args.scheme
-        n_pages = min(4, w.n_layers) * w.pages_per_layer   # layers 0-3: about 10 s of single-thread CPU work
+        n_pages = min(4, b.L) * w.pages_per_layer   # layers 0-3: about 10 s of single-thread CPU work
         src = oracle_pages(w, n_pages, True)
         tc, td, nbytes = oracle_sample(w, src)
         out["cpu_baseline"] = {"value": 2 * nbytes / (tc + td) / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
@@ -750,6 +911,10 @@ def main():
             out["cpu_baseline"]["all_cores"] = {"value": 2 * nb / (tcm + tdm) / 1e9, "unit": "GB/s", "cores": cores,
                                                 "compress_gbs": nb / tcm / 1e9, "gather_gbs": nb / tdm / 1e9,
                                                 "sample": f"the same pages, {nb >> 20} MiB split over {cores} threads, one pool each"}
+    if world == 1 and not args.no_workloads and w.name == "llama2-70b-gqa" and not args.layers:
+        free_cuda(b)
+        del b
+        out["workloads"] = other_workloads(args, dev, peak)
     print(json.dumps(out), flush=True)
     if world > 1:
         dist.destroy_process_group()

@@ -212,7 +212,14 @@ int speckv_decompress_gather_host(speckv_ctx *ctx, uint32_t layer, const int32_t
  * entry whose record is not inside the pool is reported (SPECKV_ST_BAD_RECORD, index = slot) and
  * cleared.  scratch: DEVICE memory, 256-byte aligned, at least speckv_compact_scratch_bytes(ctx)
  * bytes (pool_bytes + 4 bytes per slot + a little), contents undefined afterwards.  Prefetch
- * residency tags stay valid (they name blocks, not offsets). */
+ * residency tags stay valid (they name blocks, not offsets).
+ *
+ * speckv_free_slots gives slots back (a finished request's blocks): the listed page-table entries are
+ * cleared, so the slots read as never written and their records are garbage that the next speckv_compact
+ * drops.  freed (DEVICE uint64[2], optional, added to): [0] entries that were valid, [1] the 64-byte units
+ * their records occupy.  A slot listed twice counts once; slots[i] beyond the table is reported as
+ * SPECKV_ST_BAD_INDEX with index i.  Prefetch-buffer tags of the freed blocks are the caller's to clear. */
+int speckv_free_slots(speckv_ctx *ctx, const uint32_t *slots, uint32_t n, uint64_t *freed, void *stream);
 uint64_t speckv_compact_scratch_bytes(speckv_ctx *ctx);
 int speckv_compact(speckv_ctx *ctx, void *scratch, uint64_t scratch_bytes, void *stream);
 
@@ -245,6 +252,31 @@ int speckv_attend_dense(speckv_ctx *ctx, const void *kv, const uint32_t *seq_len
 int speckv_decompress_attend(speckv_ctx *ctx, uint32_t layer, const int32_t *block_table, const uint32_t *seq_lens,
                              uint32_t B, const void *q, uint32_t n_q_heads, void *out, void *workspace,
                              uint64_t workspace_bytes, void *stream);
+
+/* Multi-layer pipelined prefetch (Sec. 3.4.4: "while computing layer l, prefetch for layers l+1 and l+2",
+ * T_effective = T_compute + max(T_prefetch - 2 T_layer, 0)).  The call owns the schedule: a fetch stream
+ * of the context runs speckv_decompress_gather for layers layer0 .. layer0+n_layers-1 into a ring of
+ * ring_slots demand workspaces (slot r = ring + r*slot_tokens*2*H*128*2 bytes, each with room for
+ * slot_tokens token rows; 3 slots = the layer in use and two ahead), and for each layer, once its pages
+ * are there, calls consume(user, layer, slot, stream), which enqueues that layer's computation on `stream`
+ * and returns 0 (anything else ends the call and is returned).  A slot is refilled only after the
+ * computation that read it has finished; the first gather starts after the work already enqueued on
+ * `stream`.  Everything is enqueued; the call returns without synchronising.  On return, work enqueued on
+ * `stream` follows all of it.  The first call on a context creates the fetch stream and its events (no
+ * device memory) and should come before any stream capture.  seq_lens, dst_tok_off, block_table as for
+ * speckv_decompress_gather (one set for all layers); no prefetch list.
+ *
+ * speckv_pipeline_attend is the same with the library's own per-layer computation, decode-step attention
+ * over the fetched workspace:  q, out  fp16 [n_layers][B][n_q_heads][128]; workspace as for
+ * speckv_attend_dense (shared by the layers, which run one after the other on `stream`). */
+typedef int (*speckv_layer_fn)(void *user, uint32_t layer, const void *kv, void *stream);
+int speckv_pipeline_layers(speckv_ctx *ctx, uint32_t layer0, uint32_t n_layers, const int32_t *block_table,
+                           const uint32_t *seq_lens, const uint64_t *dst_tok_off, uint32_t B, void *ring,
+                           uint32_t ring_slots, uint64_t slot_tokens, speckv_layer_fn consume, void *user, void *stream);
+int speckv_pipeline_attend(speckv_ctx *ctx, uint32_t layer0, uint32_t n_layers, const int32_t *block_table,
+                           const uint32_t *seq_lens, const uint64_t *dst_tok_off, uint32_t B, void *ring,
+                           uint32_t ring_slots, uint64_t slot_tokens, const void *q, uint32_t n_q_heads, void *out,
+                           void *workspace, uint64_t workspace_bytes, void *stream);
 
 /* Managed prefetch buffer: the paper's tier L2 with its double buffering (Sec. 3.3.1), its handling
  * of mispredictions (Sec. 3.4.3: lazy invalidation, fallback to a synchronous fetch, prefetch depth

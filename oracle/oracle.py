@@ -190,6 +190,14 @@ class Pool:
         return lib().okv_compact(C.byref(self.cfg), _p(self.pool), _p(self.pte), C.byref(self.cursor), _p(scratch),
                                  C.byref(self.status))
 
+    def free_slots(self, slots):
+        """Clears the listed entries; returns [entries freed, granules released] of this call."""
+        sl = _arr(slots, np.uint32)
+        freed = np.zeros(2, np.uint64)
+        rc = lib().okv_free_slots(C.byref(self.cfg), _p(self.pte), _p(sl), C.c_uint32(sl.size), _p(freed), C.byref(self.status))
+        assert rc == 0
+        return [int(freed[0]), int(freed[1])]
+
     def translate(self, block_table, va):
         bt = _arr(block_table, np.int32)
         va = np.ascontiguousarray(va, dtype=VADDR)

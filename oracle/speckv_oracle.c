@@ -423,6 +423,25 @@ int okv_compact(const okv_config *cfg, uint8_t *pool, uint64_t *pte, uint64_t *c
     return 0;
 }
 
+/* Slot free (pool lifecycle): the listed slots' page-table entries are cleared; their records stay in
+ * the log as garbage until the next compaction.  freed[0] += entries that were valid, freed[1] += the
+ * granules their records occupy.  A slot named twice counts once; a slot beyond the table is reported
+ * (BAD_INDEX, index = position in the list). */
+int okv_free_slots(const okv_config *cfg, uint64_t *pte, const uint32_t *slots, uint32_t n,
+                   uint64_t *freed, okv_status *st)
+{
+    for (uint32_t i = 0; i < n; ++i) {
+        if (slots[i] >= n_slots(cfg)) { raise_status(st, OKV_ST_BAD_INDEX, i); continue; }
+        uint64_t e = pte[slots[i]];
+        pte[slots[i]] = 0;
+        if (!((e >> 56) & 1u)) continue;
+        uint32_t rec_len = (uint32_t)((e >> 32) & 0xFFFFu);
+        freed[0] += 1;
+        freed[1] += (rec_len + GRANULE - 1u) / GRANULE;
+    }
+    return 0;
+}
+
 /* Address translation: (seq, layer, K|V, head, token position) -> page slot -> record.
  * Layer-major regions; inside a layer the 2*H pages of one physical block are adjacent. */
 static int walk(const okv_config *cfg, const uint64_t *pte, const int32_t *block_table,

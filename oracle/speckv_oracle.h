@@ -99,6 +99,8 @@ int okv_compress(const okv_config *cfg, uint8_t *pool, uint64_t *pte, uint64_t *
  * no page-table entry points at and packs the rest in slot order.  scratch: pool_bytes bytes. */
 int okv_compact(const okv_config *cfg, uint8_t *pool, uint64_t *pte, uint64_t *cursor64,
                 uint8_t *scratch, okv_status *st);
+int okv_free_slots(const okv_config *cfg, uint64_t *pte, const uint32_t *slots, uint32_t n,
+                   uint64_t *freed, okv_status *st);
 int okv_translate(const okv_config *cfg, const uint64_t *pte, const int32_t *block_table,
                   const okv_vaddr *va, okv_paddr *pa, uint32_t n, okv_status *st);
 int okv_decompress_gather(const okv_config *cfg, const uint8_t *pool, const uint64_t *pte,

@@ -32,7 +32,12 @@ EXPORTS = ["speckv_create", "speckv_destroy", "speckv_reset", "speckv_compress",
            "speckv_attend_workspace_bytes", "speckv_attend_dense", "speckv_decompress_attend",
            "speckv_compact_scratch_bytes", "speckv_compact", "speckv_prefetch_step", "speckv_get_status", "speckv_get_stats", "speckv_clear_status", "speckv_pool_ptr",
            "speckv_pte_ptr", "speckv_l2_tag_ptr", "speckv_get_cursor", "speckv_version",
-           "speckv_set_wait_limits", "speckv_inject_missing_tiles", "speckv_set_gather_chaining"]
+           "speckv_set_wait_limits", "speckv_inject_missing_tiles", "speckv_set_gather_chaining", "speckv_free_slots",
+           "speckv_pipeline_layers", "speckv_pipeline_attend"]
+
+
+# speckv_layer_fn: int consume(void *user, uint32_t layer, const void *kv, void *stream)
+LAYER_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p)
 
 
 class SpeckvError(RuntimeError):
@@ -89,6 +94,9 @@ def load_library(path: str = LIB_PATH):
     lib.speckv_set_wait_limits.argtypes = [vp, u32, u64]
     lib.speckv_inject_missing_tiles.argtypes = [vp, u32]
     lib.speckv_set_gather_chaining.argtypes = [vp, i32]
+    lib.speckv_free_slots.argtypes = [vp, vp, u32, vp, vp]
+    lib.speckv_pipeline_layers.argtypes = [vp, u32, u32, vp, vp, vp, u32, vp, u32, u64, LAYER_FN, vp, vp]
+    lib.speckv_pipeline_attend.argtypes = [vp, u32, u32, vp, vp, vp, u32, vp, u32, u64, vp, u32, vp, vp, u64, vp]
     lib.speckv_get_cursor.argtypes = [vp, C.POINTER(u64), vp]
     for name in ("speckv_pool_ptr", "speckv_pte_ptr", "speckv_l2_tag_ptr"):
         getattr(lib, name).argtypes = [vp]
@@ -207,6 +215,12 @@ class Context:
             _ptr(dst_tok_off, (torch.int64,), "dst_tok_off"), B, _ptr(pf), n_pf, _ptr(dst_demand), cap, _ptr(dst_l2),
             _stream()), "speckv_decompress_gather")
 
+    def free_slots(self, slots, freed=None):
+        """speckv_free_slots: slots int32 tensor (read as uint32); freed int64[2] tensor or None (added to)."""
+        import torch
+        _check(self._lib.speckv_free_slots(self._h, _ptr(slots, (torch.int32,), "slots"), int(slots.numel()),
+                                           _ptr(freed, (torch.int64,), "freed"), _stream()), "speckv_free_slots")
+
     def compact_scratch_bytes(self) -> int:
         return int(self._lib.speckv_compact_scratch_bytes(self._h))
 
@@ -254,6 +268,48 @@ class Context:
             self._h, layer, _ptr(block_table, (torch.int32,), "block_table"), _ptr(seq_lens, (torch.int32,), "seq_lens"),
             B, _ptr(q, (torch.float16,), "q"), n_q_heads, _ptr(out, (torch.float16,), "out"),
             _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()), "speckv_decompress_attend")
+
+    def _ring_args(self, ring, ring_slots):
+        H = self.cfg.n_kv_heads
+        slot_tokens = ring.numel() * ring.element_size() // ring_slots // (2 * H * 256)
+        if slot_tokens == 0:
+            raise SpeckvError("ring too small")
+        return slot_tokens
+
+    def pipeline_layers(self, layer0: int, n_layers: int, block_table, seq_lens, dst_tok_off, ring, ring_slots: int, consume):
+        """speckv_pipeline_layers: gathers run up to ring_slots - 1 layers ahead on the context's fetch stream;
+        consume(layer, kv_ptr, stream_ptr) is called per layer and enqueues that layer's work on the current stream."""
+        import torch
+        failed = []
+
+        def trampoline(_user, layer, kv, stream):
+            try:
+                consume(int(layer), int(kv), int(stream or 0))
+                return 0
+            except Exception as exc:                      # an exception must not cross the C frames
+                failed.append(exc)
+                return -1
+
+        fn = LAYER_FN(trampoline)
+        rc = self._lib.speckv_pipeline_layers(
+            self._h, layer0, n_layers, _ptr(block_table, (torch.int32,), "block_table"), _ptr(seq_lens, (torch.int32,), "seq_lens"),
+            _ptr(dst_tok_off, (torch.int64,), "dst_tok_off"), int(seq_lens.numel()), _ptr(ring), ring_slots,
+            self._ring_args(ring, ring_slots), fn, None, _stream())
+        if failed:
+            raise failed[0]
+        _check(rc, "speckv_pipeline_layers")
+
+    def pipeline_attend(self, layer0: int, n_layers: int, block_table, seq_lens, dst_tok_off, ring, ring_slots: int, q, out,
+                        workspace):
+        """speckv_pipeline_attend: q, out fp16 [n_layers][B][n_q_heads][128]."""
+        import torch
+        B = int(seq_lens.numel())
+        n_q_heads = q.numel() // (n_layers * B * 128)
+        _check(self._lib.speckv_pipeline_attend(
+            self._h, layer0, n_layers, _ptr(block_table, (torch.int32,), "block_table"), _ptr(seq_lens, (torch.int32,), "seq_lens"),
+            _ptr(dst_tok_off, (torch.int64,), "dst_tok_off"), B, _ptr(ring), ring_slots, self._ring_args(ring, ring_slots),
+            _ptr(q, (torch.float16,), "q"), n_q_heads, _ptr(out, (torch.float16,), "out"), _ptr(workspace),
+            workspace.numel() * workspace.element_size(), _stream()), "speckv_pipeline_attend")
 
     def compress_host(self, src_host, staging, src_page, dst_slot, scheme: int = INT8_DELTA_RLE):
         """speckv_compress_host: src_host is a (pinned) CPU tensor of pages, staging a CUDA tensor of the same size."""

@@ -145,6 +145,36 @@ __global__ void __launch_bounds__(256) compact_copy_back_kernel(CompactArgs a)
         dst[i] = src[i];
 }
 
+// speckv_free_slots: one thread per list entry swaps the page-table entry for zero; what it found there
+// decides what is counted, so a slot named twice counts once whatever the scheduling.
+__global__ void __launch_bounds__(256) free_slots_kernel(unsigned long long *pte, unsigned long long n_slots, Ctl *ctl,
+                                                        const uint32_t *slots, uint32_t n, unsigned long long *freed)
+{
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    uint32_t entries = 0, gran = 0;
+    if (i < n) {
+        const uint32_t slot = slots[i];
+        if (slot >= n_slots) raise_status(ctl, SPECKV_ST_BAD_INDEX, i);
+        else {
+            const unsigned long long e = atomicExch(&pte[slot], 0ull);
+            if (e & kPteValid) { entries = 1; gran = (((uint32_t)(e >> 32) & 0xFFFFu) + kGranule - 1u) / kGranule; }
+        }
+    }
+    entries = __reduce_add_sync(kFull, entries);
+    gran = __reduce_add_sync(kFull, gran);
+    if ((threadIdx.x & 31u) == 0 && entries && freed) {
+        atomicAdd(&freed[0], (unsigned long long)entries);
+        atomicAdd(&freed[1], (unsigned long long)gran);
+    }
+}
+
+cudaError_t launch_free_slots(unsigned long long *pte, unsigned long long n_slots, Ctl *ctl, const uint32_t *slots, uint32_t n,
+                              unsigned long long *freed, cudaStream_t stream)
+{
+    free_slots_kernel<<<(n + 255u) / 256u, 256, 0, stream>>>(pte, n_slots, ctl, slots, n, freed);
+    return cudaGetLastError();
+}
+
 size_t compact_scratch_bytes(unsigned long long n_slots, unsigned long long pool_bytes)
 {
     const unsigned long long n_blocks = (n_slots + kCBlock - 1) / kCBlock;

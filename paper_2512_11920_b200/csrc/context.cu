@@ -29,6 +29,11 @@ struct speckv_ctx {
     int n_span;
     bool chain_live, chain_skipped, chain_enabled;
     cudaStream_t chain_stream;
+    // speckv_pipeline_layers: the fetch stream and one pair of events per ring slot (made at the first call)
+    static constexpr uint32_t kMaxRing = 8;
+    cudaStream_t fetch_stream;
+    cudaEvent_t ev_start, ev_fetched[kMaxRing], ev_consumed[kMaxRing];
+    bool pipeline_ready;
 };
 
 // How the next gather may be launched (GatherArgs::chain), and the bookkeeping for the one after.
@@ -92,6 +97,7 @@ int speckv_create(speckv_ctx **out, const speckv_config *cfg)
     c->n_slots = (unsigned long long)cfg->n_layers * cfg->blocks_per_layer * 2ull * cfg->n_kv_heads;
     c->epoch = 0;
     c->n_span = 0; c->chain_live = false; c->chain_skipped = false; c->chain_stream = nullptr; c->chain_enabled = true;
+    c->pipeline_ready = false;
     c->spin_limit = kDefaultSpinLimit;
     c->wait_ns = kDefaultWaitNs;
     c->missing_tiles = 0;
@@ -115,6 +121,11 @@ int speckv_create(speckv_ctx **out, const speckv_config *cfg)
 int speckv_destroy(speckv_ctx *c)
 {
     if (!c) return SPECKV_E_ARG;
+    if (c->pipeline_ready) {
+        cudaStreamDestroy(c->fetch_stream);
+        cudaEventDestroy(c->ev_start);
+        for (uint32_t i = 0; i < speckv_ctx::kMaxRing; ++i) { cudaEventDestroy(c->ev_fetched[i]); cudaEventDestroy(c->ev_consumed[i]); }
+    }
     cudaFree(c->pool);
     cudaFree(c->pte);
     cudaFree(c->l2_tag);
@@ -269,6 +280,16 @@ int speckv_compact(speckv_ctx *c, void *scratch, uint64_t scratch_bytes, void *s
                           (cudaStream_t)stream) == cudaSuccess ? 0 : SPECKV_E_CUDA;
 }
 
+int speckv_free_slots(speckv_ctx *c, const uint32_t *slots, uint32_t n, uint64_t *freed, void *stream)
+{
+    if (!c) return SPECKV_E_ARG;
+    if (n == 0) return 0;
+    if (!slots || ((uintptr_t)slots & 3u) || ((uintptr_t)freed & 7u)) return SPECKV_E_ARG;
+    c->chain_live = false;
+    return launch_free_slots(c->pte, c->n_slots, c->ctl, slots, n, (unsigned long long *)freed, (cudaStream_t)stream) == cudaSuccess
+               ? 0 : SPECKV_E_CUDA;
+}
+
 // ---- decode-step attention over fetched pages
 
 static size_t attend_prefix_bytes(uint32_t B) { return (((size_t)B + 1) * 4 + 255) & ~(size_t)255; }
@@ -316,6 +337,86 @@ int speckv_decompress_attend(speckv_ctx *c, uint32_t layer, const int32_t *block
     a.pool = c->pool; a.pte = c->pte; a.block_table = block_table; a.pool_bytes = c->cfg.pool_bytes;
     a.layer = layer; a.blocks_per_layer = c->cfg.blocks_per_layer; a.max_blocks_per_seq = c->cfg.max_blocks_per_seq;
     return attend_common(c, a, true, seq_lens, B, q, n_q_heads, out, workspace, workspace_bytes, stream);
+}
+
+// ---- multi-layer pipelined prefetch (Sec. 3.4.4)
+
+static int pipeline_setup(speckv_ctx *c)
+{
+    if (c->pipeline_ready) return 0;
+    if (cudaStreamCreateWithFlags(&c->fetch_stream, cudaStreamNonBlocking) != cudaSuccess) return SPECKV_E_CUDA;
+    bool ok = cudaEventCreateWithFlags(&c->ev_start, cudaEventDisableTiming) == cudaSuccess;
+    for (uint32_t i = 0; i < speckv_ctx::kMaxRing; ++i)
+        ok = ok && cudaEventCreateWithFlags(&c->ev_fetched[i], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&c->ev_consumed[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) return SPECKV_E_CUDA;
+    c->pipeline_ready = true;
+    return 0;
+}
+
+int speckv_pipeline_layers(speckv_ctx *c, uint32_t layer0, uint32_t n_layers, const int32_t *block_table,
+                           const uint32_t *seq_lens, const uint64_t *dst_tok_off, uint32_t B, void *ring,
+                           uint32_t ring_slots, uint64_t slot_tokens, speckv_layer_fn consume, void *user, void *stream)
+{
+    if (!c || !consume || !ring || ((uintptr_t)ring & 15u) || ring_slots < 1 || ring_slots > speckv_ctx::kMaxRing ||
+        (uint64_t)layer0 + n_layers > c->cfg.n_layers || B > c->cfg.max_seqs)
+        return SPECKV_E_ARG;
+    if (n_layers == 0) return 0;
+    int rc = pipeline_setup(c);
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream, fs = c->fetch_stream;
+    const uint64_t slot_bytes = slot_tokens * 2ull * c->cfg.n_kv_heads * SPECKV_HEAD_DIM * 2ull;
+    // the fetch stream starts after whatever the caller has enqueued so far (the writes of the pages, say)
+    if (cudaEventRecord(c->ev_start, st) != cudaSuccess || cudaStreamWaitEvent(fs, c->ev_start, 0) != cudaSuccess) return SPECKV_E_CUDA;
+    for (uint32_t l = 0; l < n_layers; ++l) {
+        const uint32_t r = l % ring_slots;
+        uint8_t *slot = (uint8_t *)ring + (uint64_t)r * slot_bytes;
+        if (l >= ring_slots) {
+            // the slot is free once the computation of the layer that used it has finished; a gather that
+            // follows an event wait is launched as an ordinary, fully ordered kernel
+            if (cudaStreamWaitEvent(fs, c->ev_consumed[r], 0) != cudaSuccess) return SPECKV_E_CUDA;
+            c->chain_live = false;
+        }
+        rc = speckv_decompress_gather(c, layer0 + l, block_table, seq_lens, dst_tok_off, B, nullptr, 0, slot, slot_tokens, nullptr, fs);
+        if (rc) return rc;
+        if (cudaEventRecord(c->ev_fetched[r], fs) != cudaSuccess || cudaStreamWaitEvent(st, c->ev_fetched[r], 0) != cudaSuccess)
+            return SPECKV_E_CUDA;
+        rc = consume(user, layer0 + l, slot, stream);
+        if (rc) return rc;
+        if (cudaEventRecord(c->ev_consumed[r], st) != cudaSuccess) return SPECKV_E_CUDA;
+    }
+    c->chain_live = false;
+    return 0;
+}
+
+struct PipelineAttend {
+    speckv_ctx *c;
+    const uint32_t *seq_lens;
+    const uint64_t *tok_off;
+    uint32_t B, n_q_heads, layer0;
+    const uint8_t *q;
+    uint8_t *out;
+    void *workspace;
+    uint64_t workspace_bytes;
+};
+static int pipeline_attend_layer(void *user, uint32_t layer, const void *kv, void *stream)
+{
+    const PipelineAttend *p = (const PipelineAttend *)user;
+    const uint64_t per_layer = (uint64_t)p->B * p->n_q_heads * SPECKV_HEAD_DIM * 2ull;
+    return speckv_attend_dense(p->c, kv, p->seq_lens, p->tok_off, p->B, p->q + (layer - p->layer0) * per_layer, p->n_q_heads,
+                               p->out + (layer - p->layer0) * per_layer, p->workspace, p->workspace_bytes, stream);
+}
+
+int speckv_pipeline_attend(speckv_ctx *c, uint32_t layer0, uint32_t n_layers, const int32_t *block_table,
+                           const uint32_t *seq_lens, const uint64_t *dst_tok_off, uint32_t B, void *ring, uint32_t ring_slots,
+                           uint64_t slot_tokens, const void *q, uint32_t n_q_heads, void *out, void *workspace,
+                           uint64_t workspace_bytes, void *stream)
+{
+    if (!c || !q || !out) return SPECKV_E_ARG;
+    PipelineAttend p = {c, seq_lens, (const uint64_t *)dst_tok_off, B, n_q_heads, layer0, (const uint8_t *)q, (uint8_t *)out,
+                        workspace, workspace_bytes};
+    return speckv_pipeline_layers(c, layer0, n_layers, block_table, seq_lens, dst_tok_off, B, ring, ring_slots, slot_tokens,
+                                  pipeline_attend_layer, &p, stream);
 }
 
 // ---- managed prefetch buffer

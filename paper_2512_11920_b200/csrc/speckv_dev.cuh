@@ -174,6 +174,8 @@ uint32_t attend_max_warps();
 size_t compact_scratch_bytes(unsigned long long n_slots, unsigned long long pool_bytes);
 cudaError_t launch_compact(uint8_t *pool, unsigned long long pool_bytes, unsigned long long *pte, unsigned long long n_slots,
                            Ctl *ctl, uint8_t *scratch, int n_sm, cudaStream_t stream);
+cudaError_t launch_free_slots(unsigned long long *pte, unsigned long long n_slots, Ctl *ctl, const uint32_t *slots, uint32_t n,
+                              unsigned long long *freed, cudaStream_t stream);
 cudaError_t launch_gather(const GatherArgs &a, int n_sm, cudaStream_t stream);
 cudaError_t launch_translate(const TranslateArgs &a, cudaStream_t stream);
 uint32_t compress_tile_pages(int scheme);

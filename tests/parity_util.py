@@ -86,6 +86,15 @@ class Pair:
                                      f"worst distance {worst} ulp; tolerance is 1 ulp and bit-exact is expected")
         return d_got, l_got
 
+    def free_slots(self, slots):
+        slots = np.asarray(slots, np.uint32)
+        want = self.cpu.free_slots(slots)
+        freed = self.torch.zeros(2, dtype=self.torch.int64, device=self.dev)
+        self.gpu.free_slots(self.t(slots), freed)
+        got = [int(v) for v in freed.cpu().numpy()]
+        assert got == want, f"freed {got} != {want}"
+        return got
+
     def compact(self):
         self.cpu.compact()
         # zeroed like the oracle's: when shared records overflow the pool, the granules between the last copy

@@ -46,8 +46,8 @@ def test_compaction_over_many_blocks_with_rewrites_raw_pages_and_bad_entries():
     again = rng.permutation(len(slots))[:700]
     pr.compress(w.gen_pages(slots), again, slots[again], 0)                        # a third of layer 1 rewritten raw
     victims = rng.permutation(w.n_slots)[:5]
+    assert pr.free_slots([victims[0]])[0] == 1                                     # a freed slot
     for pte in (pr.cpu.pte, pr.gpu.pte_view().view(pr.torch.int64)):
-        pte[int(victims[0])] = 0                                                   # freed slot
         pte[int(victims[1])] = (int(pr.cpu.cfg.pool_bytes // 64) - 1) | (4112 << 32) | (1 << 56)   # ends beyond the pool
         pte[int(victims[2])] = 5 | (9 << 32) | (1 << 56)                           # shorter than a header
     pr.compact()
@@ -94,4 +94,30 @@ def test_entries_sharing_records_overflow_the_pool():
     assert pr.gpu.cursor() == 2 * used and 0 < st["count"][O.ST_POOL_FULL] < len(slots)
     live = int((pr.cpu.pte >> 56 & 1).sum())
     assert live == 2 * len(slots) - st["count"][O.ST_POOL_FULL]
+    pr.close()
+
+
+def test_free_slots_then_compaction_reclaims_a_finished_sequence():
+    """A request ends: every slot of its blocks is freed (some named twice, one out of range), the counts
+    equal the oracle's, gathers of the other sequences are unchanged, the freed one reads as never written,
+    and compaction shrinks the log by exactly the granules that were reported."""
+    w = workloads.llama70b(seed=21, n_layers=2, batch=3, seq=320)                  # 20 blocks per sequence
+    pr = Pair.for_workload(w, pool_bytes=w.n_slots * 4160)
+    for layer in range(2):
+        slots = w.layer_slots(layer)
+        pr.compress(w.gen_pages(slots), np.arange(len(slots)), slots, 3 if layer else 0)
+    before = pr.gpu.cursor()
+    gone = np.concatenate([w.layer_slots(layer, blocks=w.block_table[1]) for layer in range(2)])
+    listed = np.concatenate([gone, gone[:40], [w.n_slots + 7]]).astype(np.uint32)
+    entries, gran = pr.free_slots(listed)
+    assert entries == len(gone) == 2 * 20 * 16
+    pr.check_state()
+    st = pr.gpu.status()
+    assert st["count"][O.ST_BAD_INDEX] == 1 and st["first"][O.ST_BAD_INDEX] == len(listed) - 1
+    for layer in range(2):
+        pr.gather(layer, w.block_table, w.seq_lens, w.dst_tok_off())              # sequence 1: BAD_PTE, left untouched
+    assert pr.gpu.status()["count"][O.ST_BAD_PTE] == len(gone)
+    pr.compact()
+    pr.check_state()
+    assert pr.gpu.cursor() == before - gran
     pr.close()

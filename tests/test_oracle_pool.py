@@ -441,3 +441,23 @@ def test_gather_skips_a_sequence_whose_rows_pass_the_destination_capacity():
     dst2 = np.full(80 * 2 * H * 128, 0xCDCD, np.uint16)
     assert pool.decompress_gather(0, w.block_table, w.seq_lens[:2], np.array([0, 48], np.uint64), None, dst2, l2) == 0
     assert sum(pool.status_dict()["count"]) == 0 and not np.any(np.all(dst2.reshape(-1, 2048) == 0xCDCD, axis=1))
+
+
+def test_free_slots_clears_entries_and_counts_what_compaction_will_reclaim():
+    """Worked by hand: an all-zero page (5 granules) in slot 0, a constant page (5) in slot 2, a raw page (65) in
+    slot 5.  Freeing [2, 7, 2, 99, 5]: slot 2 once (5 granules), slot 7 was empty, 99 is beyond the 8 slots
+    (reported at list position 3), slot 5 (65 granules) -> 2 entries, 70 granules; compaction then keeps
+    slot 0 alone."""
+    pool = O.Pool(1, 1, 4, 4, 1, 64 * 200)
+    zero, const = np.zeros(2048, np.uint16), _h(np.full(2048, 3.5))
+    pool.compress(np.stack([zero, const]), [0, 1], [0, 2], 3)
+    pool.compress(np.stack([const]), [0], [5], 0)
+    assert pool.cursor.value == 75
+    assert pool.free_slots([2, 7, 2, 99, 5]) == [2, 70]
+    st = pool.status_dict()
+    assert st["count"][O.ST_BAD_INDEX] == 1 and st["first"][O.ST_BAD_INDEX] == 3 and sum(st["count"]) == 1
+    assert [bool(e >> 56 & 1) for e in pool.pte] == [True] + [False] * 7
+    assert pool.cursor.value == 75                                  # the log itself is untouched
+    assert pool.compact() == 0 and pool.cursor.value == 5
+    assert pool.free_slots([0, 0]) == [1, 5] and not pool.pte.any()
+    assert pool.compact() == 0 and pool.cursor.value == 0
