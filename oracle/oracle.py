@@ -233,6 +233,44 @@ class Pool:
         return out
 
 
+N_CANDIDATES = 8
+CANDIDATE_SCHEMES = (1, 2, 3, 4, 17, 18, 19, 20)
+PROBE = np.dtype([("pages", "<u8"), ("nonfinite", "<u8"), ("bad_index", "<u8"), ("granules", "<u8", (8,)),
+                  ("sq_err", "<f8", (2,)), ("sq_sum", "<f8")])
+POLICY = np.dtype([("w_r", "<f8"), ("w_q", "<f8"), ("w_c", "<f8"), ("q_min", "<f8"), ("cost", "<f8", (8,))])
+
+
+def probe_pages(src_bits, src_page, probe=None):
+    """Adds what the listed pages cost and lose under every candidate scheme to `probe` (a PROBE record)."""
+    src = _arr(src_bits, np.uint16).reshape(-1, PAGE_ELEMS)
+    sp = _arr(src_page, np.uint32)
+    out = np.zeros(1, PROBE) if probe is None else np.ascontiguousarray(probe, dtype=PROBE).reshape(1)
+    rc = lib().okv_probe_pages(_p(src), C.c_uint32(src.shape[0]), _p(sp), C.c_uint32(sp.size), _p(out))
+    assert rc == 0
+    return out
+
+
+def make_policy(w_r, w_q, w_c, q_min, cost):
+    pol = np.zeros(1, POLICY)
+    pol["w_r"], pol["w_q"], pol["w_c"], pol["q_min"] = w_r, w_q, w_c, q_min
+    pol["cost"][0] = cost
+    return pol
+
+
+def probe_quality(probe, grouped: bool) -> float:
+    lib().okv_probe_quality.restype = C.c_double
+    pr = np.ascontiguousarray(probe, dtype=PROBE).reshape(1)
+    return float(lib().okv_probe_quality(_p(pr), C.c_int(int(grouped))))
+
+
+def select_scheme(probe, policy):
+    """(scheme, J of the 8 candidates) for one layer's probe and a policy."""
+    pr = np.ascontiguousarray(probe, dtype=PROBE).reshape(1)
+    pol = np.ascontiguousarray(policy, dtype=POLICY).reshape(1)
+    obj = np.zeros(N_CANDIDATES, np.float64)
+    return int(lib().okv_select_scheme(_p(pr), _p(pol), _p(obj))), obj
+
+
 def pf_score(reward: int, plays: int, steps: int, beta: float) -> float:
     """The depth rule's score of one arm: mean reward + exploration bonus."""
     return float(lib().okv_pf_score(int(reward), int(plays), int(steps), float(beta)))

@@ -442,6 +442,80 @@ int okv_free_slots(const okv_config *cfg, uint64_t *pte, const uint32_t *slots, 
     return 0;
 }
 
+/* ---------------------------------------------------------------------- */
+/* Compression selection per layer (Sec. 3.6.3):                            */
+/*   C*(l,t) = argmax_{C in CC} J,  J = w_r R_c(C,l) + w_q Q(C,l) - w_c L_comp(C),  s.t. Q >= Q_min */
+/* ---------------------------------------------------------------------- */
+
+/* The candidate set CC, in the order that breaks ties (simpler first). */
+static const int probe_schemes[OKV_N_CANDIDATES] = {
+    OKV_INT8, OKV_INT8_DELTA, OKV_INT8_DELTA_RLE, OKV_AUTO,
+    OKV_INT8 | OKV_GROUPED, OKV_INT8_DELTA | OKV_GROUPED, OKV_INT8_DELTA_RLE | OKV_GROUPED, OKV_AUTO | OKV_GROUPED};
+
+/* What a sample of a layer's pages would cost and lose under every candidate: each page is really
+ * compressed with each scheme (size) and the two quantisers' records are really decompressed (error).
+ * Pages holding Inf/NaN are stored raw whatever the scheme and are only counted. */
+int okv_probe_pages(const uint16_t *src, uint32_t n_src_pages, const uint32_t *src_page, uint32_t n,
+                    okv_probe *out)
+{
+    uint8_t rec[HDR_BYTES + PAGE_BYTES + GRANULE];
+    uint16_t back[PAGE_ELEMS];
+    for (uint32_t i = 0; i < n; ++i) {
+        if (src_page[i] >= n_src_pages) { out->bad_index += 1; continue; }
+        const uint16_t *x = src + (uint64_t)src_page[i] * PAGE_ELEMS;
+        uint32_t len = okv_compress_page(x, PAGE_N, PAGE_D, OKV_INT8, rec);
+        if (rec[6] == OKV_RAW) { out->nonfinite += 1; continue; }
+        out->pages += 1;
+        for (int c = 0; c < OKV_N_CANDIDATES; ++c) {
+            len = okv_compress_page(x, PAGE_N, PAGE_D, probe_schemes[c], rec);
+            out->granules[c] += (len + GRANULE - 1u) / GRANULE;
+        }
+        for (int g = 0; g < 2; ++g) {   /* the lossy step is the quantiser: one scale per page, or per group */
+            len = okv_compress_page(x, PAGE_N, PAGE_D, g ? (OKV_INT8 | OKV_GROUPED) : OKV_INT8, rec);
+            okv_decompress_record(rec, len, PAGE_N, PAGE_D, back);
+            for (uint32_t k = 0; k < PAGE_ELEMS; ++k) {
+                double e = (double)okv_half_to_float(x[k]) - (double)okv_half_to_float(back[k]);
+                out->sq_err[g] += e * e;
+            }
+        }
+        for (uint32_t k = 0; k < PAGE_ELEMS; ++k) {
+            double v = (double)okv_half_to_float(x[k]);
+            out->sq_sum += v * v;
+        }
+    }
+    return 0;
+}
+
+/* Quality Q of a quantiser on the sample: signal-to-noise ratio in decibels, capped at 200 (also
+ * when there is no error at all). */
+double okv_probe_quality(const okv_probe *p, int grouped)
+{
+    double err = p->sq_err[grouped ? 1 : 0];
+    if (!(err > 0.0) || !(p->sq_sum > 0.0)) return 200.0;
+    double q = 10.0 * log10(p->sq_sum / err);
+    return q > 200.0 ? 200.0 : q;
+}
+
+/* The selection itself.  R_c = uncompressed bytes / stored bytes of the sample.  Among the candidates
+ * with Q >= q_min the largest J wins, the earlier candidate on a tie; if no candidate reaches q_min, the
+ * one with the best quality does (earlier on a tie).  objective (optional): J of every candidate.
+ * Returns the scheme, or -1 if the sample is empty. */
+int okv_select_scheme(const okv_probe *p, const okv_policy *pol, double *objective)
+{
+    if (p->pages == 0) return -1;
+    int best = -1, best_q = 0;
+    double best_j = 0.0;
+    for (int c = 0; c < OKV_N_CANDIDATES; ++c) {
+        double ratio = (double)p->pages * (double)(PAGE_BYTES / GRANULE) / (double)p->granules[c];
+        double q = okv_probe_quality(p, c >= 4);
+        double j = pol->w_r * ratio + pol->w_q * q - pol->w_c * pol->cost[c];
+        if (objective) objective[c] = j;
+        if (q >= pol->q_min && (best < 0 || j > best_j)) { best = c; best_j = j; }
+        if (q > okv_probe_quality(p, best_q >= 4)) best_q = c;
+    }
+    return probe_schemes[best >= 0 ? best : best_q];
+}
+
 /* Address translation: (seq, layer, K|V, head, token position) -> page slot -> record.
  * Layer-major regions; inside a layer the 2*H pages of one physical block are adjacent. */
 static int walk(const okv_config *cfg, const uint64_t *pte, const int32_t *block_table,

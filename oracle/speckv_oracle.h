@@ -99,6 +99,25 @@ int okv_compress(const okv_config *cfg, uint8_t *pool, uint64_t *pte, uint64_t *
  * no page-table entry points at and packs the rest in slot order.  scratch: pool_bytes bytes. */
 int okv_compact(const okv_config *cfg, uint8_t *pool, uint64_t *pte, uint64_t *cursor64,
                 uint8_t *scratch, okv_status *st);
+/* ---- compression selection per layer (Sec. 3.6.3) ----------------------- */
+/* The paper gives the form  C*(l,t) = argmax_C  w_r R_c(C,l) + w_q Q(C,l) - w_c L_comp(C)  s.t. Q >= Q_min
+ * and leaves the candidate set, Q and L_comp open.  Here: candidates = schemes 1-4 with one scale per
+ * page, then the same four with one scale per channel group; R_c = stored ratio on a sample of the
+ * layer's pages; Q = signal-to-quantisation-noise ratio of the sample in dB; L_comp and the weights are
+ * the caller's numbers. */
+enum { OKV_N_CANDIDATES = 8 };
+typedef struct {
+    uint64_t pages, nonfinite, bad_index; /* pages measured / skipped (Inf, NaN) / list entries out of range */
+    uint64_t granules[OKV_N_CANDIDATES];  /* 64-byte granules the measured pages take under each candidate */
+    double sq_err[2];                     /* sum of (x - decoded x)^2: page scale, grouped scales */
+    double sq_sum;                        /* sum of x^2 */
+} okv_probe;
+typedef struct { double w_r, w_q, w_c, q_min; double cost[OKV_N_CANDIDATES]; } okv_policy;
+int okv_probe_pages(const uint16_t *src, uint32_t n_src_pages, const uint32_t *src_page, uint32_t n,
+                    okv_probe *out);
+double okv_probe_quality(const okv_probe *p, int grouped);
+int okv_select_scheme(const okv_probe *p, const okv_policy *pol, double *objective);
+
 int okv_free_slots(const okv_config *cfg, uint64_t *pte, const uint32_t *slots, uint32_t n,
                    uint64_t *freed, okv_status *st);
 int okv_translate(const okv_config *cfg, const uint64_t *pte, const int32_t *block_table,
