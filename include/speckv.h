@@ -253,6 +253,38 @@ int speckv_decompress_attend(speckv_ctx *ctx, uint32_t layer, const int32_t *blo
                              uint32_t B, const void *q, uint32_t n_q_heads, void *out, void *workspace,
                              uint64_t workspace_bytes, void *stream);
 
+/* Compression selection per layer (Sec. 3.6.3, policy engine):
+ *     C*(l,t) = argmax_{C in CC}  w_r R_c(C,l) + w_q Q(C,l) - w_c L_comp(C)    subject to  Q(C,l) >= Q_min.
+ * The paper leaves CC, Q and L_comp open.  Here CC = the schemes 1, 2, 3, 4 with one scale per page followed
+ * by the same four with SPECKV_GROUPED (candidate index 0..7, the order that breaks ties); R_c = uncompressed
+ * bytes / stored bytes (64-byte units) of a sample of the layer's pages; Q = signal-to-quantisation-noise
+ * ratio of that sample in decibels, 10 log10(sum x^2 / sum (x - decoded x)^2), capped at 200; L_comp(C) and
+ * the weights are the caller's numbers (the paper updates its weights by gradient steps on a throughput
+ * reward that only a serving system has).
+ *
+ * speckv_probe_pages measures the sample on the GPU: page i of the list is read from src + 4096*src_page[i],
+ * quantised with both scale granularities, its delta symbols' run heads are counted, and `out` (DEVICE, zeroed
+ * by the caller before the first call for a layer, added to by every call) receives what the pages would
+ * occupy under each candidate and the squared errors.  Pages holding Inf or NaN (stored raw by every scheme)
+ * and list entries >= n_src_pages are only counted.  Stateless: needs no context.  Integer fields are exact;
+ * the three sums are binary64 sums of exact terms in an unspecified order.
+ *
+ * speckv_select_scheme (HOST arithmetic, binary64; probe and policy in HOST memory) returns the scheme to
+ * pass to speckv_compress for that layer: the candidate with the largest objective among those with
+ * Q >= q_min, the earlier one on a tie; if none qualifies, the earliest candidate of the best quality.
+ * objective (optional, HOST double[8]) receives every candidate's value.  SPECKV_E_ARG for an empty sample. */
+#define SPECKV_N_CANDIDATES 8
+typedef struct {
+    uint64_t pages, nonfinite, bad_index;    /* measured / skipped for Inf, NaN / list entries out of range */
+    uint64_t granules[SPECKV_N_CANDIDATES];  /* 64-byte units the measured pages take under each candidate  */
+    double sq_err[2];                        /* sum (x - decoded x)^2: one scale per page, per channel group */
+    double sq_sum;                           /* sum x^2                                                     */
+} speckv_probe;
+typedef struct { double w_r, w_q, w_c, q_min; double cost[SPECKV_N_CANDIDATES]; } speckv_policy;
+int speckv_probe_pages(const void *src, uint32_t n_src_pages, const uint32_t *src_page, uint32_t n, speckv_probe *out,
+                       void *stream);
+int speckv_select_scheme(const speckv_probe *probe, const speckv_policy *policy, double *objective);
+
 /* Multi-layer pipelined prefetch (Sec. 3.4.4: "while computing layer l, prefetch for layers l+1 and l+2",
  * T_effective = T_compute + max(T_prefetch - 2 T_layer, 0)).  The call owns the schedule: a fetch stream
  * of the context runs speckv_decompress_gather for layers layer0 .. layer0+n_layers-1 into a ring of

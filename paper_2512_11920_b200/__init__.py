@@ -5,4 +5,5 @@ include/speckv.h); `binding` marshals torch tensors into it.  There is no CPU fa
 the library is missing or the device is not a B200-class GPU, calls raise.
 """
 from .binding import (Context, SpeckvError, PREFETCH_DTYPE, VADDR_DTYPE, PADDR_DTYPE, load_library,  # noqa: F401
-                      RAW, INT8, INT8_DELTA, INT8_DELTA_RLE, AUTO, GROUPED, compress_static, STATIC_MAX_PAGES, CTL_BLOCK_BYTES)
+                      RAW, INT8, INT8_DELTA, INT8_DELTA_RLE, AUTO, GROUPED, compress_static, STATIC_MAX_PAGES, CTL_BLOCK_BYTES,
+                      probe_pages, select_scheme, PROBE_DTYPE, CANDIDATE_SCHEMES)

@@ -33,7 +33,7 @@ EXPORTS = ["speckv_create", "speckv_destroy", "speckv_reset", "speckv_compress",
            "speckv_compact_scratch_bytes", "speckv_compact", "speckv_prefetch_step", "speckv_get_status", "speckv_get_stats", "speckv_clear_status", "speckv_pool_ptr",
            "speckv_pte_ptr", "speckv_l2_tag_ptr", "speckv_get_cursor", "speckv_version",
            "speckv_set_wait_limits", "speckv_inject_missing_tiles", "speckv_set_gather_chaining", "speckv_free_slots",
-           "speckv_pipeline_layers", "speckv_pipeline_attend"]
+           "speckv_pipeline_layers", "speckv_pipeline_attend", "speckv_probe_pages", "speckv_select_scheme"]
 
 
 # speckv_layer_fn: int consume(void *user, uint32_t layer, const void *kv, void *stream)
@@ -95,6 +95,8 @@ def load_library(path: str = LIB_PATH):
     lib.speckv_inject_missing_tiles.argtypes = [vp, u32]
     lib.speckv_set_gather_chaining.argtypes = [vp, i32]
     lib.speckv_free_slots.argtypes = [vp, vp, u32, vp, vp]
+    lib.speckv_probe_pages.argtypes = [vp, u32, vp, u32, vp, vp]
+    lib.speckv_select_scheme.argtypes = [vp, vp, vp]
     lib.speckv_pipeline_layers.argtypes = [vp, u32, u32, vp, vp, vp, u32, vp, u32, u64, LAYER_FN, vp, vp]
     lib.speckv_pipeline_attend.argtypes = [vp, u32, u32, vp, vp, vp, u32, vp, u32, u64, vp, u32, vp, vp, u64, vp]
     lib.speckv_get_cursor.argtypes = [vp, C.POINTER(u64), vp]
@@ -157,6 +159,38 @@ def compress_static(src, src_page, dst_slot, scheme, pool, pte, ctl):
                                       n, scheme, _ptr(pool, (torch.uint8,), "pool"), pool.numel(),
                                       _ptr(pte, (torch.int64,), "pte"), pte.numel(), _ptr(ctl), _stream()),
            "speckv_compress_static")
+
+
+PROBE_DTYPE = np.dtype([("pages", "<u8"), ("nonfinite", "<u8"), ("bad_index", "<u8"), ("granules", "<u8", (8,)),
+                        ("sq_err", "<f8", (2,)), ("sq_sum", "<f8")])
+POLICY_DTYPE = np.dtype([("w_r", "<f8"), ("w_q", "<f8"), ("w_c", "<f8"), ("q_min", "<f8"), ("cost", "<f8", (8,))])
+CANDIDATE_SCHEMES = (1, 2, 3, 4, 17, 18, 19, 20)
+
+
+def probe_pages(src, src_page, probe):
+    """speckv_probe_pages: adds the measurements of the listed pages to `probe`, a zeroed uint8 CUDA tensor of
+    PROBE_DTYPE.itemsize bytes (one layer's accumulator)."""
+    import torch
+    lib = load_library()
+    if probe.numel() * probe.element_size() < PROBE_DTYPE.itemsize:
+        raise SpeckvError("probe too small")
+    _check(lib.speckv_probe_pages(_ptr(src, None, "src"), src.numel() * src.element_size() // 4096,
+                                  _ptr(src_page, (torch.int32,), "src_page"), int(src_page.numel()), _ptr(probe), _stream()),
+           "speckv_probe_pages")
+
+
+def select_scheme(probe, w_r: float, w_q: float, w_c: float, q_min: float, cost):
+    """speckv_select_scheme: probe = a PROBE_DTYPE record on the host (numpy); returns (scheme, objective[8])."""
+    lib = load_library()
+    pr = np.ascontiguousarray(probe, dtype=PROBE_DTYPE).reshape(1)
+    pol = np.zeros(1, POLICY_DTYPE)
+    pol["w_r"], pol["w_q"], pol["w_c"], pol["q_min"] = w_r, w_q, w_c, q_min
+    pol["cost"][0] = cost
+    obj = np.zeros(8, np.float64)
+    rc = lib.speckv_select_scheme(pr.ctypes.data_as(C.c_void_p), pol.ctypes.data_as(C.c_void_p), obj.ctypes.data_as(C.c_void_p))
+    if rc < 0:
+        _check(rc, "speckv_select_scheme")
+    return int(rc), obj
 
 
 class Context:

@@ -8,7 +8,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libspeckv.so")
-SOURCES = ["context.cu", "compress.cu", "gather.cu", "attend.cu", "compact.cu", "prefetch.cu"]
+SOURCES = ["context.cu", "compress.cu", "gather.cu", "attend.cu", "compact.cu", "prefetch.cu", "policy.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
               "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 
