@@ -229,6 +229,7 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src)
 __global__ void __launch_bounds__(kDWarps * 32, 3) attend_dense_kernel(AttendArgs a)
 {
     extern __shared__ __align__(16) uint8_t smem[];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");          // the merge kernel may be scheduled behind this grid
     uint32_t *s_blk = reinterpret_cast<uint32_t *>(smem + kDWarps * 4 * kTileBytes);
     const uint32_t tid = threadIdx.x, lane = tid & 31u;
     const uint32_t warp = __shfl_sync(kFull, tid >> 5, 0);
@@ -284,6 +285,7 @@ constexpr uint32_t kFWarpBytes = 2 * kFStage + 2 * kTileBytes;
 __global__ void __launch_bounds__(kFWarps * 32, 2) attend_fused_kernel(AttendArgs a)
 {
     extern __shared__ __align__(16) uint8_t smem[];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");          // the merge kernel may be scheduled behind this grid
     uint32_t *s_lut = reinterpret_cast<uint32_t *>(smem + kFWarps * kFWarpBytes);          // [256]
     unsigned long long *s_bar = reinterpret_cast<unsigned long long *>(s_lut + 256);      // [kFWarps][2]
     uint32_t *s_blk = reinterpret_cast<uint32_t *>(s_bar + kFWarps * 2);
@@ -411,6 +413,9 @@ __global__ void __launch_bounds__(kFWarps * 32, 2) attend_fused_kernel(AttendArg
 // S = prefix[b]*H + h*nblk, so its partials come from the warps S/per .. (S + nblk - 1)/per.
 __global__ void __launch_bounds__(128) attend_combine_kernel(AttendArgs a, uint32_t n_warps)
 {
+    // launched while the attention kernel is still running (programmatic dependent launch): its blocks are
+    // resident and past their set-up when the last partial result lands
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t wid = blockIdx.x * 4u + (threadIdx.x >> 5), Hq = a.H * a.G;
     if (wid >= a.B * Hq) return;
@@ -473,7 +478,18 @@ cudaError_t launch_attend(const AttendArgs &a, bool fused, int n_sm, cudaStream_
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const uint32_t n_out = a.B * a.H * a.G;
-    if (n_out) attend_combine_kernel<<<(n_out + 3u) / 4u, 128, 0, stream>>>(a, n_warps);
+    if (n_out) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((n_out + 3u) / 4u);
+        cfg.blockDim = dim3(128);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // see griddepcontrol.wait in the kernel
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, attend_combine_kernel, a, n_warps);
+    }
     return cudaGetLastError();
 }
 

@@ -3,7 +3,7 @@
 // adapted per request) and the depth rule of Sec. 3.6.3 (upper confidence bound over depths 1..4).
 //
 // Two launches per call:
-//   pf_plan_kernel   one thread per sequence: looks this step's reads up in the readable bank, scores
+//   pf_plan_kernel   four threads per sequence (one per depth score): looks this step's reads up in the readable bank, scores
 //                    the fill that is about to be overwritten, picks the depth, retags the slots of the
 //                    bank being filled.  Everything that touches tags and statistics happens here, in a
 //                    fixed order per sequence, so the outcome does not depend on scheduling.
@@ -38,11 +38,18 @@ __device__ __forceinline__ double depth_score(int reward, uint32_t plays, uint32
     return __dadd_rn(mean, bonus);
 }
 
-__global__ void __launch_bounds__(128) pf_plan_kernel(PrefetchArgs a)
+__global__ void __launch_bounds__(32) pf_plan_kernel(PrefetchArgs a)
 {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the fetch kernel may start its set-up
-    const uint32_t b = blockIdx.x * blockDim.x + threadIdx.x;
+    // Four threads per sequence.  All four walk the sequence's (short) bookkeeping alike, so that each holds
+    // the updated statistics; the four depth scores — a binary64 logarithm, square root and two divisions
+    // each, the long pole of this kernel — are then evaluated side by side, one per thread.  Only the first
+    // thread of a quad reports, counts and stores.
+    const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t b = t >> 2, arm = t & 3u;
+    const bool lead = arm == 0;
     const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t live = __ballot_sync(kFull, b < a.B);   // whole quads: the lanes that take part in the shuffles below
     unsigned long long n_acc = 0, n_hit = 0, n_late = 0, n_miss = 0, n_fetch = 0, n_kept = 0, n_evict = 0, n_evict_used = 0;
     if (b < a.B) {
         speckv_pf_seq s = a.state[b];
@@ -57,7 +64,8 @@ __global__ void __launch_bounds__(128) pf_plan_kernel(PrefetchArgs a)
             wh[i] = -2;
             if (acc[i] < 0) continue;
             if ((uint32_t)acc[i] >= a.max_blocks_per_seq) {
-                for (uint32_t r = 0; r < twoH; ++r) raise_status(a.ctl, SPECKV_ST_UNMAPPED, (b * 4u + i) * twoH + r);
+                if (lead)
+                    for (uint32_t r = 0; r < twoH; ++r) raise_status(a.ctl, SPECKV_ST_UNMAPPED, (b * 4u + i) * twoH + r);
                 continue;
             }
             const uint32_t tag = a.layer * (1u << 20) + (uint32_t)acc[i] + 1u;
@@ -79,7 +87,7 @@ __global__ void __launch_bounds__(128) pf_plan_kernel(PrefetchArgs a)
                 wh[i] = -1;
             }
         }
-        reinterpret_cast<int4 *>(a.where)[b] = make_int4(wh[0], wh[1], wh[2], wh[3]);
+        if (lead) reinterpret_cast<int4 *>(a.where)[b] = make_int4(wh[0], wh[1], wh[2], wh[3]);
         // 2. score the fill that is about to be overwritten
         const uint32_t d = s.depth[back];
         if (d > 0) {
@@ -94,13 +102,16 @@ __global__ void __launch_bounds__(128) pf_plan_kernel(PrefetchArgs a)
         uint32_t k = 0;
         for (uint32_t j = 0; j < 4 && !k; ++j)
             if (s.plays[j] == 0) k = j + 1;
+        // (every thread of the quad takes this branch or none does: they hold the same statistics)
+        const double mine = k ? 0.0 : depth_score(s.reward[arm], s.plays[arm], s.steps, a.beta);
+        double sc[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) sc[j] = __shfl_sync(live, mine, j, 4);
         if (!k) {
             k = 1;
-            double best = depth_score(s.reward[0], s.plays[0], s.steps, a.beta);
-            for (uint32_t j = 1; j < 4; ++j) {
-                const double sc = depth_score(s.reward[j], s.plays[j], s.steps, a.beta);
-                if (sc > best) { best = sc; k = j + 1; }
-            }
+            double best = sc[0];
+            for (uint32_t j = 1; j < 4; ++j)
+                if (sc[j] > best) { best = sc[j]; k = j + 1; }                 // ties: the smaller depth
         }
         // 4. retag the slots of the bank being filled; the transfers follow in pf_fetch_kernel
         uint32_t fill = 0;
@@ -109,7 +120,8 @@ __global__ void __launch_bounds__(128) pf_plan_kernel(PrefetchArgs a)
             if (cb < 0 || (uint32_t)cb >= a.max_blocks_per_seq) continue;
             const int32_t p = __ldg(a.block_table + (size_t)b * a.max_blocks_per_seq + (uint32_t)cb);
             if (p < 0 || (uint32_t)p >= a.blocks_per_layer) {
-                for (uint32_t r = 0; r < twoH; ++r) raise_status(a.ctl, SPECKV_ST_UNMAPPED, ((a.B + b) * 4u + j) * twoH + r);
+                if (lead)
+                    for (uint32_t r = 0; r < twoH; ++r) raise_status(a.ctl, SPECKV_ST_UNMAPPED, ((a.B + b) * 4u + j) * twoH + r);
                 continue;
             }
             const uint32_t tag = a.layer * (1u << 20) + (uint32_t)cb + 1u;
@@ -122,8 +134,9 @@ __global__ void __launch_bounds__(128) pf_plan_kernel(PrefetchArgs a)
         }
         s.fill = (uint8_t)fill;
         s.depth[back] = (uint8_t)k;
-        a.state[b] = s;
+        if (lead) a.state[b] = s;
     }
+    if (!lead) n_acc = n_hit = n_late = n_miss = n_fetch = n_kept = n_evict = n_evict_used = 0;
     unsigned long long v[8] = {n_acc, n_hit, n_late, n_miss, n_fetch, n_kept, n_evict, n_evict_used};
     unsigned long long *out = reinterpret_cast<unsigned long long *>(a.cnt);
 #pragma unroll
@@ -292,7 +305,7 @@ static size_t pf_fetch_smem(uint32_t B)
 
 cudaError_t launch_prefetch_step(const PrefetchArgs &a, int n_sm, cudaStream_t stream)
 {
-    pf_plan_kernel<<<(a.B + 127u) / 128u, 128, 0, stream>>>(a);
+    pf_plan_kernel<<<(a.B + 7u) / 8u, 32, 0, stream>>>(a);   // one warp = eight sequences
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const size_t smem = pf_fetch_smem(a.B);

@@ -173,11 +173,17 @@ class Pair:
             bad = np.nonzero(pte != self.cpu.pte)[0]
             raise AssertionError(f"{bad.size} page-table entries differ, first slot {bad[0]}: "
                                  f"{int(pte[bad[0]]):#x} != {int(self.cpu.pte[bad[0]]):#x}")
-        used = min(cur * 64, self.cpu.cfg.pool_bytes)
-        pool = self.gpu.pool_view(max(used, 1)).cpu().numpy()[:used]
-        if not np.array_equal(pool, self.cpu.pool[:used]):
-            bad = np.nonzero(pool != self.cpu.pool[:used])[0]
-            raise AssertionError(f"compressed bytestream differs in {bad.size} bytes, first at byte {bad[0]}")
+        # The whole pool, not only the log up to the cursor: bytes behind the cursor are a canary (nothing may be
+        # written there; after a compaction they keep what the old log held, on both sides alike).  Pools too
+        # large to copy whole are compared up to the cursor and on 64 MiB behind it.
+        total = self.cpu.cfg.pool_bytes
+        used = min(cur * 64, total)
+        upto = total if total <= (1 << 28) else min(total, used + (64 << 20))
+        pool = self.gpu.pool_view(upto).cpu().numpy()
+        if not np.array_equal(pool, self.cpu.pool[:upto]):
+            bad = np.nonzero(pool != self.cpu.pool[:upto])[0]
+            where = "compressed bytestream" if bad[0] < used else "pool bytes behind the cursor (nothing may be written there)"
+            raise AssertionError(f"{where}: {bad.size} bytes differ, first at byte {bad[0]} (cursor at byte {used})")
         tags = self.gpu.l2_tag_view().cpu().numpy().view(np.uint64)
         assert np.array_equal(tags, self.cpu.l2_tag), "prefetch tags differ"
         assert self.gpu.stats() == self.cpu.stats.as_dict(), f"{self.gpu.stats()} != {self.cpu.stats.as_dict()}"
