@@ -236,6 +236,19 @@ __device__ __forceinline__ uint4 encode_page(const uint4 *in, int scheme, bool g
             for (int k = 0; k < 8; ++k) pay[k * 32 + lane] = make_uint2(q[k][0], q[k][1]);
         } else {
             mode = SPECKV_INT8_DELTA_RLE;
+            // (first, so that these stores are under way while the scan below waits for its shuffles)
+            wait_rec();
+            // zero the value area and the padding (values are OR-ed in), store the bitmap
+            {
+                uint4 *z = reinterpret_cast<uint4 *>(rec + kValuesOff);
+                constexpr uint32_t n16max = (kRecSlot - kValuesOff) / 16;
+                const uint32_t n16 = n16max - grp / 16u;     // up to the end of this warp's staging slot
+#pragma unroll
+                for (uint32_t jj = 0; jj < (n16max + 31u) / 32u; ++jj)
+                    if (jj * 32u + lane < n16) z[jj * 32u + lane] = make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) rec[kHdrBytes + k * 32 + lane] = (uint8_t)mk[k];
             // ---- offset of each group's run values: exclusive prefix sum of the popcounts in (k, lane)
             // order.  Within a group row the exclusive sums stay below 8 * 31 = 248, so four rows share a
             // word as byte fields and nothing carries between them; the row totals (up to 256) are warp
@@ -251,18 +264,6 @@ __device__ __forceinline__ uint4 encode_page(const uint4 *in, int scheme, bool g
                 excl[k] = __byte_perm(k < 4 ? ea : eb, 0u, 0x4440 + (k & 3));
                 tot[k] = __reduce_add_sync(kFull, c[k]);
             }
-            wait_rec();
-            // zero the value area and the padding (values are OR-ed in), store the bitmap
-            {
-                uint4 *z = reinterpret_cast<uint4 *>(rec + kValuesOff);
-                constexpr uint32_t n16max = (kRecSlot - kValuesOff) / 16;
-                const uint32_t n16 = n16max - grp / 16u;     // up to the end of this warp's staging slot
-#pragma unroll
-                for (uint32_t jj = 0; jj < (n16max + 31u) / 32u; ++jj)
-                    if (jj * 32u + lane < n16) z[jj * 32u + lane] = make_uint4(0u, 0u, 0u, 0u);
-            }
-#pragma unroll
-            for (int k = 0; k < 8; ++k) rec[kHdrBytes + k * 32 + lane] = (uint8_t)mk[k];
             __syncwarp();
             // ---- compaction: head bytes moved to the front of the group (PRMT), shifted to the byte
             // offset inside their words, OR-ed into the staged value stream
