@@ -104,8 +104,9 @@ class ClockSampler:
 class Bench:
     """Device-resident state of one replica: source K/V, context, index tensors, destination."""
 
-    def __init__(self, w, dev, scheme=3, layer0=0, n_layers=None):
-        """Layers [layer0, layer0 + n_layers) of workload w (default: all); the context numbers them from 0."""
+    def __init__(self, w, dev, scheme=3, layer0=0, n_layers=None, pool_page_bytes=4160):
+        """Layers [layer0, layer0 + n_layers) of workload w (default: all); the context numbers them from 0.
+        pool_page_bytes: pool capacity per page (4,160 = every page stored raw; 2,368 = the largest packed record)."""
         import torch
         from kvgen import device as gen_device
         from paper_2512_11920_b200 import Context
@@ -117,7 +118,7 @@ class Bench:
         self.scales = torch.from_numpy(w.scales).to(dev)
         for l in range(self.L):
             gen_device.fill(self.src[l * ppl * 2048:(l + 1) * ppl * 2048], w.seed, (layer0 + l) * ppl, ppl, self.scales, ppl, w.n_kv_heads)
-        pool_bytes = ((self.pages * 4160 + (64 << 20)) // 64) * 64          # room for every page stored raw
+        pool_bytes = ((self.pages * pool_page_bytes + (64 << 20)) // 64) * 64
         self.ctx = Context(self.L, w.n_kv_heads, w.blocks_per_layer, w.max_blocks_per_seq, w.batch, pool_bytes)
         # compress lists a layer's pages in physical slot order (source and page table share the numbering)
         self.idx_all = torch.arange(self.pages, dtype=torch.int32, device=dev)

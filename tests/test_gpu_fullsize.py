@@ -6,7 +6,9 @@ layer).
 The oracle cannot process 20 GiB in a test, so: (a) sampled pages are compared bit for bit
 (record bytes, page-table entry, gathered fp16), (b) properties that hold at any size are
 checked over ALL pages on the device (placement = prefix sum in list order, every page
-delivered, nothing reported)."""
+delivered, nothing reported), (c) idempotence over ALL pages: the gathered K/V of every layer is
+compressed again and must give the first pass's records byte for byte (the oracle's pinned property
+compress(decompress(C)) == C), so a rare wrong page in either direction cannot hide among the unsampled."""
 import numpy as np
 import pytest
 
@@ -25,11 +27,11 @@ def test_full_size_sampled_parity_and_placement(name, layers, scheme):
     import bench
     from kvgen import workloads
     w = workloads.BY_NAME[name](seed=0, n_layers=layers)
-    need = 2.7 * w.n_slots * 4096 / 2 ** 30
+    need = (2.6 + 0.6 / layers) * w.n_slots * 4096 / 2 ** 30
     torch.cuda.empty_cache()                                                     # blocks cached from earlier tests count as used
     if _free_gib() < need + 4:
         pytest.skip(f"needs {need:.0f} GiB of free device memory")
-    b = bench.Bench(w, torch.device("cuda:0"), scheme)
+    b = bench.Bench(w, torch.device("cuda:0"), scheme, pool_page_bytes=2368)
     grp = 32 if scheme & 16 else 0                                               # bytes of group maxima per record
     b.dst.fill_(-1)
     b.step()
@@ -53,6 +55,31 @@ def test_full_size_sampled_parity_and_placement(name, layers, scheme):
     # (a) sampled pages against the oracle
     res = b.sampled_parity(n_samples=64, seed=7)
     assert res["mismatches"] == 0, res
+    # (c) idempotence, every page of every layer: where slot s of the layer sits in the gathered workspace
+    from paper_2512_11920_b200 import Context
+    H, ppl = w.n_kv_heads, w.pages_per_layer
+    nblk = (w.seq_lens.astype(np.int64) + 15) // 16
+    tok = w.dst_tok_off().astype(np.int64)
+    where = np.full(ppl, -1, np.int64)
+    for s_ in range(w.batch):
+        p = w.block_table[s_, :nblk[s_]].astype(np.int64)                         # physical blocks of the sequence, in logical order
+        for kv in range(2):
+            for h in range(H):
+                where[(p * 2 + kv) * H + h] = tok[s_] * 2 * H // 16 + (kv * H + h) * nblk[s_] + np.arange(nblk[s_])
+    assert (where >= 0).all()
+    again = Context(1, H, w.blocks_per_layer, w.max_blocks_per_seq, w.batch, ((ppl * 2368 + (1 << 20)) // 64) * 64)
+    src_page = torch.from_numpy(where.astype(np.int32)).cuda()
+    slots = torch.arange(ppl, dtype=torch.int32, device="cuda")
+    pool1 = b.ctx.pool_view()
+    for l in range(w.n_layers):
+        again.reset()
+        again.compress(b.dst_layer(l), src_page, slots, scheme)
+        n64 = again.cursor()
+        first = int(pte[l * ppl].item()) & 0xFFFFFFFF
+        assert torch.equal(again.pool_view(n64 * 64), pool1[first * 64:(first + n64) * 64]), f"layer {l}: recompressed records differ"
+        assert torch.equal(again.pte_view().view(torch.int64) + first, pte[l * ppl:(l + 1) * ppl]), f"layer {l}: entries differ"
+    assert sum(again.status()["count"]) == 0
+    again.close()
     b.ctx.close()
 
 
@@ -68,7 +95,7 @@ def test_repeated_fast_scheme_runs_keep_every_record():
     torch.cuda.empty_cache()
     if _free_gib() < 2.7 * w.n_slots * 4096 / 2 ** 30 + 4:
         pytest.skip("needs 54 GiB of free device memory")
-    b = bench.Bench(w, torch.device("cuda:0"), 4)
+    b = bench.Bench(w, torch.device("cuda:0"), 4, pool_page_bytes=2368)
     nan = torch.tensor([0x7E00], dtype=torch.int16, device="cuda")
     for page in (5, 2_000_003, b.pages - 9, b.pages - 4):                       # raw pages, two of them in the last tiles
         b.src[page * 2048 + 77] = nan[0]
