@@ -109,7 +109,10 @@ typedef struct {
 
 /* Creates a context on the current device: allocates (cudaMalloc) and zeroes the pool
  * (pool_bytes), the page table (8 B per slot), the prefetch tags and small control blocks.
- * Synchronises the device.  cfg is HOST memory.  Fails with SPECKV_E_DEVICE on a GPU that is
+ * Synchronises the device.  cfg is HOST memory.  Limits (SPECKV_E_ARG beyond): n_kv_heads <= 255,
+ * n_layers <= 4095, blocks_per_layer and max_blocks_per_seq < 2^20, max_seqs <= 4096,
+ * max_seqs*max_blocks_per_seq*2*n_kv_heads < 2^31 (page indices are 32-bit), pool_bytes a multiple of 64
+ * below 2^38.  Fails with SPECKV_E_DEVICE on a GPU that is
  * not sm_100.  speckv_destroy frees everything the context allocated. */
 int speckv_create(speckv_ctx **out, const speckv_config *cfg);
 int speckv_destroy(speckv_ctx *ctx);
@@ -157,7 +160,11 @@ int speckv_translate(speckv_ctx *ctx, const int32_t *block_table, const speckv_v
  *   dst_tok_off[b]*2*H*128 + ((kv*H + head)*Tpad_b + 16*n)*128,  Tpad_b = 16*ceil(seq_lens[b]/16)
  * i.e. each sequence is a dense [2][H][Tpad_b][128] fp16 tensor starting at token row
  * dst_tok_off[b] (the caller normally passes the exclusive prefix sum of Tpad).  A sequence
- * whose rows would pass dst_cap_tokens is skipped (SPECKV_ST_BAD_DST).
+ * whose rows would pass dst_cap_tokens is skipped (SPECKV_ST_BAD_DST).  A sequence longer than the
+ * block table can describe (more than max_blocks_per_seq blocks) is reported once as
+ * SPECKV_ST_UNMAPPED, at the page index its first page would have had, and left out altogether: none of
+ * its pages is fetched and it takes no place in the page numbering (speckv_decompress_attend likewise:
+ * its output rows are zero).
  * Prefetch part (the loop of the prefetching algorithm after token prediction): entry e
  * names logical block pf[e].block of sequence pf[e].seq; if the prefetch-buffer slot
  * (seq, l2_slot) is already tagged with this (layer, block) the entry is skipped, otherwise

@@ -588,7 +588,10 @@ int okv_decompress_gather(const okv_config *cfg, const uint8_t *pool, const uint
      * heads.  Sequence b owns Tpad_b = 16*ceil(len_b/16) token rows starting at dst_tok_off[b];
      * inside it the layout is [K|V][head][token][channel]. */
     for (uint32_t b = 0; b < B; ++b) {
-        uint32_t nblk = (seq_lens[b] + PAGE_N - 1u) / PAGE_N;
+        uint32_t nblk = (uint32_t)(((uint64_t)seq_lens[b] + PAGE_N - 1u) / PAGE_N);
+        /* a length the block table cannot describe: the sequence is reported once, at the index its
+         * first page would have had, and takes no part (no pages, no place in the numbering) */
+        if (nblk > cfg->max_blocks_per_seq) { raise_status(st, OKV_ST_UNMAPPED, index); continue; }
         uint64_t tpad = (uint64_t)nblk * PAGE_N;
         for (uint32_t n = 0; n < nblk; ++n)
             for (uint32_t kv = 0; kv < 2u; ++kv)
@@ -699,7 +702,12 @@ int okv_attend(const okv_config *cfg, const uint8_t *pool, const uint64_t *pte, 
     uint32_t index0 = 0; /* page index of the sequence's first page, numbered as in the demand fetch */
     for (uint32_t b = 0; b < B; ++b) {
         uint32_t len = seq_lens[b];
-        uint32_t nblk = (len + PAGE_N - 1u) / PAGE_N;
+        uint32_t nblk = (uint32_t)(((uint64_t)len + PAGE_N - 1u) / PAGE_N);
+        if (nblk > cfg->max_blocks_per_seq) { /* as in the demand fetch: reported once, left out, zero output */
+            raise_status(st, OKV_ST_UNMAPPED, index0);
+            for (uint64_t i = 0; i < (uint64_t)Hq * PAGE_D; ++i) out[(uint64_t)b * Hq * PAGE_D + i] = 0.0;
+            continue;
+        }
         uint16_t *kpage = (uint16_t *)malloc((size_t)(nblk + 1u) * PAGE_BYTES);
         uint16_t *vpage = (uint16_t *)malloc((size_t)(nblk + 1u) * PAGE_BYTES);
         const uint16_t **kr = (const uint16_t **)malloc((len + 1u) * sizeof(*kr));

@@ -154,9 +154,14 @@ __device__ __forceinline__ void attn_end(AttnState &st, float *partial, uint32_t
 
 // s_blk[b] = number of 16-token blocks of the sequences before b (shared memory, [B + 1]); also
 // written to the workspace for the merge pass.
-__device__ __forceinline__ void build_prefix(const AttendArgs &a, uint32_t *s_blk, uint32_t tid, uint32_t n_threads)
+// `limit`: most blocks a sequence may have (the block table's width for the fused source); a longer one is
+// reported once as unmapped, at the index its first page would have had, and contributes no blocks.
+__device__ __forceinline__ void build_prefix(const AttendArgs &a, uint32_t *s_blk, uint32_t tid, uint32_t n_threads, uint32_t limit)
 {
-    for (uint32_t b = tid; b < a.B; b += n_threads) s_blk[b + 1] = (a.seq_lens[b] + 15u) >> 4;
+    for (uint32_t b = tid; b < a.B; b += n_threads) {
+        const unsigned long long nb = ((unsigned long long)a.seq_lens[b] + 15ull) >> 4;
+        s_blk[b + 1] = nb > limit ? 0u : (uint32_t)nb;
+    }
     if (tid == 0) s_blk[0] = 0;
     __syncthreads();
     if (tid < 32) {                                       // one warp: serial over 32-wide pieces
@@ -174,8 +179,11 @@ __device__ __forceinline__ void build_prefix(const AttendArgs &a, uint32_t *s_bl
         }
     }
     __syncthreads();
-    if (blockIdx.x == 0)
+    if (blockIdx.x == 0) {
         for (uint32_t b = tid; b <= a.B; b += n_threads) a.prefix[b] = s_blk[b];
+        for (uint32_t b = tid; b < a.B; b += n_threads)
+            if ((((unsigned long long)a.seq_lens[b] + 15ull) >> 4) > limit) raise_status(a.ctl, SPECKV_ST_UNMAPPED, s_blk[b] * 2u * a.H);
+    }
 }
 
 // This warp's share [g0, g1) of the list of T = H * (all blocks) block positions, ordered by
@@ -233,7 +241,7 @@ __global__ void __launch_bounds__(kDWarps * 32, 3) attend_dense_kernel(AttendArg
     uint32_t *s_blk = reinterpret_cast<uint32_t *>(smem + kDWarps * 4 * kTileBytes);
     const uint32_t tid = threadIdx.x, lane = tid & 31u;
     const uint32_t warp = __shfl_sync(kFull, tid >> 5, 0);
-    build_prefix(a, s_blk, tid, kDWarps * 32);
+    build_prefix(a, s_blk, tid, kDWarps * 32, 0xFFFFFFFFu);   // the workspace holds what the lengths say: no table to exceed
     const uint32_t tiles = smem_u32(smem + warp * 4 * kTileBytes);          // [stage][K|V]
     const uint32_t row = lane >> 4, col = lane & 15u;                         // a 16-byte piece of a token row
     const uint32_t w = blockIdx.x * kDWarps + warp;
@@ -294,7 +302,7 @@ __global__ void __launch_bounds__(kFWarps * 32, 2) attend_fused_kernel(AttendArg
     s_lut[tid & 255u] = expand_sel(tid & 15u) | (expand_sel((tid >> 4) & 15u) << 16);
     if (tid < kFWarps * 2) mbar_init(smem_u32(s_bar + tid), 1);
     mbar_init_fence();
-    build_prefix(a, s_blk, tid, kFWarps * 32);
+    build_prefix(a, s_blk, tid, kFWarps * 32, a.max_blocks_per_seq);
     uint8_t *my = smem + warp * kFWarpBytes;
     uint8_t *my_rec = my;                                                     // [2][kFStage]
     uint8_t *my_tile = my + 2 * kFStage;                                      // [K|V][kTileBytes]

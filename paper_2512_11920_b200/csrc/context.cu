@@ -83,6 +83,7 @@ int speckv_create(speckv_ctx **out, const speckv_config *cfg)
     if (!cfg->n_layers || !cfg->n_kv_heads || !cfg->blocks_per_layer || !cfg->max_blocks_per_seq || !cfg->max_seqs ||
         cfg->n_kv_heads > 255 || cfg->n_layers > 4095 || cfg->blocks_per_layer >= (1u << 20) ||
         cfg->max_blocks_per_seq >= (1u << 20) || cfg->max_seqs > gather_max_seqs() || cfg->pool_bytes == 0 ||
+        (unsigned long long)cfg->max_seqs * cfg->max_blocks_per_seq * 2ull * cfg->n_kv_heads > 0x7FFFFFFFull ||   // page indices are 32-bit
         cfg->pool_bytes % kGranule || cfg->pool_bytes / kGranule > 0xFFFFFFFFull)
         return SPECKV_E_ARG;
     int dev = 0;

@@ -70,7 +70,12 @@ __global__ void __launch_bounds__(kGThreads, 3) gather_kernel(GatherArgs a)
     const uint32_t warp = __shfl_sync(kFull, tid >> 5, 0);                        // warp-uniform for the compiler too
     s_lut[tid & 255u] = expand_sel(tid & 15u) | (expand_sel((tid >> 4) & 15u) << 16);
     if (tid < kGWarps * 2) mbar_init(smem_u32(s_bar + tid), 1);
-    for (uint32_t b = tid; b < a.B; b += kGThreads) { s_pref[b + 1] = (a.seq_lens[b] + 15u) >> 4; s_tok[b] = a.dst_tok_off[b]; }
+    // blocks per sequence; a length that the block table cannot describe contributes none (reported below)
+    for (uint32_t b = tid; b < a.B; b += kGThreads) {
+        const uint32_t nb = (uint32_t)(((unsigned long long)a.seq_lens[b] + 15ull) >> 4);
+        s_pref[b + 1] = nb > a.max_blocks_per_seq ? 0u : nb;
+        s_tok[b] = a.dst_tok_off[b];
+    }
     if (tid == 0) s_pref[0] = 0;
     mbar_init_fence();
     __syncthreads();
@@ -84,6 +89,9 @@ __global__ void __launch_bounds__(kGThreads, 3) gather_kernel(GatherArgs a)
         __syncthreads();
     }
 
+    if (blockIdx.x == 0)      // once per launch: sequences left out, at the index their first page would have had
+        for (uint32_t b = tid; b < a.B; b += kGThreads)
+            if ((((unsigned long long)a.seq_lens[b] + 15ull) >> 4) > a.max_blocks_per_seq) raise_status(a.ctl, SPECKV_ST_UNMAPPED, s_pref[b] * 2u * a.H);
     // Unit decomposition: a unit is a logical block (demand blocks first, then prefetch entries);
     // this warp serves page r = (kv, head) of the units g0, g0 + gstep, ...  The host sizes the grid so
     // that the number of warps is a multiple of 2*H.

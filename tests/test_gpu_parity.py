@@ -396,3 +396,36 @@ def test_gather_warps_walk_several_batches_of_pages_with_faults_and_prefetch():
     st = pr.gpu.status()["count"]
     assert st[O.ST_UNMAPPED] and st[O.ST_BAD_PTE] and st[O.ST_BAD_RECORD] and pr.gpu.stats()["pf_skipped"] > 0
     pr.close()
+
+
+def test_sequences_longer_than_the_block_table_are_reported_and_left_out():
+    """Lengths beyond what the block table describes — one block too many, and an absurd value whose block count
+    would wrap a 32-bit prefix sum: each is reported once (unmapped, at its first page's index) and nothing of
+    it is written; the others are delivered; the fused attention gives zero rows for them."""
+    w = workloads.llama70b(seed=4, n_layers=1, batch=4, seq=96)
+    pr = Pair.for_workload(w)
+    slots = w.layer_slots(0)
+    pr.compress(w.gen_pages(slots), np.arange(len(slots)), slots, 3)
+    lens = np.array([48, 97, 0xFFFFFFF0, 5], np.uint32)
+    pr.gather(0, w.block_table, lens, np.array([0, 48, 48, 48], np.uint64), cap_tokens=64)
+    pr.check_state()
+    st = pr.gpu.status()
+    assert st["count"][O.ST_UNMAPPED] == 2 and st["first"][O.ST_UNMAPPED] == 3 * 16 and sum(st["count"]) == 2
+    import torch
+    q = np.random.default_rng(1).standard_normal((4, 16, 128)).astype(np.float16)
+    want = pr.cpu.attend(0, w.block_table, lens, q.view(np.uint16), 16)
+    assert not want[1].any() and not want[2].any() and want[0].any()
+    # error bound from the sequences that take part (the helper would size buffers by the absurd length)
+    valid = np.array([48, 0, 0, 5], np.uint32)
+    _, tpad, tok = pr._layout(valid)
+    d = np.zeros(int(tpad.sum()) * 2 * w.n_kv_heads * 128, np.uint16)
+    scratch = O.Pool.__new__(O.Pool)
+    scratch.__dict__.update(pr.cpu.__dict__)
+    scratch.status, scratch.stats, scratch.l2_tag = O.Status(), O.Stats(), pr.cpu.l2_tag.copy()
+    scratch.decompress_gather(0, w.block_table, valid, tok, None, d, np.zeros(w.batch * 4 * 2 * w.n_kv_heads * 2048, np.uint16))
+    ws = torch.empty(pr.gpu.attend_workspace_bytes(4), dtype=torch.uint8, device="cuda")
+    out = torch.full((4, 16, 128), float("nan"), dtype=torch.float16, device="cuda")
+    pr.gpu.decompress_attend(0, pr.t(w.block_table), pr.t(lens), pr.t(q).view(torch.float16), out, ws)
+    pr._attend_check(out.cpu().numpy(), want, pr._vmax(d, valid, tpad, tok), 2, "decompress_attend")
+    pr.check_state()
+    pr.close()

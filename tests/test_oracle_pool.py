@@ -461,3 +461,39 @@ def test_free_slots_clears_entries_and_counts_what_compaction_will_reclaim():
     assert pool.compact() == 0 and pool.cursor.value == 5
     assert pool.free_slots([0, 0]) == [1, 5] and not pool.pte.any()
     assert pool.compact() == 0 and pool.cursor.value == 0
+
+
+def test_a_sequence_longer_than_the_block_table_is_reported_once_and_left_out():
+    """Block table 6 wide; lengths 48, 16*6 + 1 (seven blocks: one too many) and 5.  The long sequence is reported
+    once as unmapped, at the index its first page would have had (3 blocks * 2 * H), and takes no place in the
+    numbering: the third sequence's missing page is numbered right behind the first sequence's pages."""
+    w = workloads.llama70b(seed=4, n_layers=1, batch=3, seq=96)
+    assert w.max_blocks_per_seq == 6
+    pool = _fill(w)
+    H = w.n_kv_heads
+    lens = np.array([48, 97, 5], np.uint32)
+    victim = ((0 * w.blocks_per_layer + w.block_table[2][0]) * 2 + 1) * H + 3          # V page, head 3, of the third sequence
+    pool.pte[victim] = 0
+    dst = np.full(64 * 2 * H * 128, 0xCDCD, np.uint16)
+    l2 = np.zeros(w.batch * 4 * 2 * H * 2048, np.uint16)
+    assert pool.decompress_gather(0, w.block_table, lens, np.array([0, 48, 48], np.uint64), None, dst, l2) == 0
+    st = pool.status_dict()
+    assert st["count"][O.ST_UNMAPPED] == 1 and st["first"][O.ST_UNMAPPED] == 3 * 2 * H
+    assert st["count"][O.ST_BAD_PTE] == 1 and st["first"][O.ST_BAD_PTE] == 3 * 2 * H + H + 3
+    assert pool.stats.pages_decoded == 4 * 2 * H - 1
+    el = 48 * 2 * H * 128                                                               # the third sequence sits at row 48
+    slot = ((0 * w.blocks_per_layer + w.block_table[2][0]) * 2 + 0) * H + 0
+    assert np.array_equal(dst[el:el + 2048], _expected_page(w, slot))
+    # exactly as wide as the table is fine; an absurd length is the same single report
+    pool.clear_status()
+    big = np.full(112 * 2 * H * 128, 0xCDCD, np.uint16)
+    assert pool.decompress_gather(0, w.block_table, np.array([96, 0xFFFFFFFF], np.uint32), np.array([0, 96], np.uint64), None, big, l2) == 0
+    st = pool.status_dict()
+    assert st["count"][O.ST_UNMAPPED] == 1 and st["first"][O.ST_UNMAPPED] == 6 * 2 * H and sum(st["count"]) == 1
+    # the attention reading of the same rule: zero rows for the sequence that is left out
+    q = np.random.default_rng(0).standard_normal((2, H, 128)).astype(np.float16)
+    pool.clear_status()
+    out = pool.attend(0, w.block_table, np.array([97, 48], np.uint32), q.view(np.uint16), H)
+    assert not out[0].any() and out[1].any()
+    st = pool.status_dict()
+    assert st["count"][O.ST_UNMAPPED] == 1 and st["first"][O.ST_UNMAPPED] == 0 and sum(st["count"]) == 1
