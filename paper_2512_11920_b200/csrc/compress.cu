@@ -54,15 +54,21 @@ constexpr uint32_t kOffAbort = kOffBar + kNumBars * 8;
 constexpr uint32_t kCompressSmem = kOffAbort + 16;
 static_assert(kCompressSmem + 1024 <= 233472, "one CTA per SM");
 
-// Compaction table entry for a run-head mask m: x, y = PRMT selectors moving the head bytes of the
-// 8 symbols to the front (x: output bytes 0-3, y: output bytes 4-7), z, w = byte masks
-// keeping the first popcount(m) bytes.
+// Compaction table entry for a run-head mask m.  The j-th head byte comes from symbol position >= j, so the
+// output bytes 4-7 only ever come from the second word: x = PRMT selector over (q0, q1) for output bytes 0-3,
+// y = PRMT selector over (q1, zero) for output bytes 4-7 with the unused positions pointing at the zero word,
+// z = byte mask keeping the first min(popcount(m), 4) bytes of the low word (w unused).
 __device__ __forceinline__ uint4 lut_entry(uint32_t m)
 {
     const uint32_t c = __popc(m);
-    const unsigned long long keep = c == 8 ? ~0ull : ((1ull << (8 * c)) - 1ull);
+    const uint32_t keep_lo = c >= 4 ? 0xFFFFFFFFu : ((1u << (8 * c)) - 1u);
     const uint32_t sel = compact_sel(m);
-    return make_uint4(sel & 0xFFFFu, sel >> 16, (uint32_t)keep, (uint32_t)(keep >> 32));
+    uint32_t y = 0;
+    for (uint32_t j = 4; j < 8; ++j) {
+        const uint32_t pos = (sel >> (4 * j)) & 15u;                  // symbol position of head j (4..7) if j < c
+        y |= (j < c ? pos - 4u : 4u) << (4 * (j - 4));                // 4 = first byte of the zero word
+    }
+    return make_uint4(sel & 0xFFFFu, y, keep_lo, 0u);
 }
 
 // two fused multiply-adds a*b + c on packed binary32 pairs (one rounding each)
@@ -274,7 +280,7 @@ __device__ __forceinline__ uint4 encode_page(const uint4 *in, int scheme, bool g
                 const uint32_t o = base + excl[k];
                 const uint4 e = lut[mk[k]];
                 const uint32_t lo = __byte_perm(q[k][0], q[k][1], e.x) & e.z;        // PRMT reads 16 selector bits
-                const uint32_t hi = __byte_perm(q[k][0], q[k][1], e.y) & e.w;
+                const uint32_t hi = __byte_perm(q[k][1], 0u, e.y);
                 const uint32_t sh = o << 3;          // funnel shifts use the low 5 bits: 8 * (o & 3)
                 const uint32_t w0 = __funnelshift_l(0u, lo, sh), w1 = __funnelshift_l(lo, hi, sh), w2 = __funnelshift_l(hi, 0u, sh);
                 const uint32_t p = vals + (o & ~3u);
