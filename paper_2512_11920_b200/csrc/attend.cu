@@ -228,22 +228,22 @@ __device__ __forceinline__ void advance(Share &sh, const uint32_t *s_blk, uint32
 // ---------------------------------------------------------------- dense source
 
 constexpr int kDWarps = 4;
-
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
+constexpr uint32_t kDStages = 2;   // K+V tile pairs per warp: the block in use and the next one on its way
 
 __global__ void __launch_bounds__(kDWarps * 32, 3) attend_dense_kernel(AttendArgs a)
 {
     extern __shared__ __align__(16) uint8_t smem[];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");          // the merge kernel may be scheduled behind this grid
-    uint32_t *s_blk = reinterpret_cast<uint32_t *>(smem + kDWarps * 4 * kTileBytes);
+    unsigned long long *s_bar = reinterpret_cast<unsigned long long *>(smem + kDWarps * kDStages * 2 * kTileBytes);   // [kDWarps][kDStages]
+    uint32_t *s_blk = reinterpret_cast<uint32_t *>(s_bar + kDWarps * kDStages);
     const uint32_t tid = threadIdx.x, lane = tid & 31u;
     const uint32_t warp = __shfl_sync(kFull, tid >> 5, 0);
+    if (tid < kDWarps * kDStages) mbar_init(smem_u32(s_bar + tid), 1);
+    mbar_init_fence();
     build_prefix(a, s_blk, tid, kDWarps * 32, 0xFFFFFFFFu);   // the workspace holds what the lengths say: no table to exceed
-    const uint32_t tiles = smem_u32(smem + warp * 4 * kTileBytes);          // [stage][K|V]
-    const uint32_t row = lane >> 4, col = lane & 15u;                         // a 16-byte piece of a token row
+    const uint32_t tiles = smem_u32(smem + warp * kDStages * 2 * kTileBytes);   // [stage][K|V]
+    const uint32_t my_bar = smem_u32(s_bar + warp * kDStages);
+    uint32_t phases = 0;                                                        // bit s: parity of stage s's barrier
     const uint32_t w = blockIdx.x * kDWarps + warp;
 
     for (Share sh = first_piece(s_blk, a.B, a.H, w, gridDim.x * kDWarps); sh.g < sh.g1;) {
@@ -254,30 +254,31 @@ __global__ void __launch_bounds__(kDWarps * 32, 3) attend_dense_kernel(AttendArg
         // workspace of the demand path: [K|V][head][token][channel] per sequence
         const uint4 *kbase = a.kv + (a.tok_off[b] * 2u * a.H * 128u + ((unsigned long long)h * tpad + 16u * n0) * 128u) / 8u;
         const uint4 *vbase = kbase + ((unsigned long long)a.H * tpad * 128u) / 8u;
-        auto load = [&](uint32_t i) {                                         // block n0 + i -> stage i & 1
-            const uint32_t dst = tiles + (i & 1u) * 2u * kTileBytes;
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const uint32_t off = (2u * k + row) * kTilePitch + col * 16u;
-                cp_async16(dst + off, kbase + (size_t)i * 256u + k * 32 + lane);
-                cp_async16(dst + kTileBytes + off, vbase + (size_t)i * 256u + k * 32 + lane);
-            }
-            asm volatile("cp.async.commit_group;" ::: "memory");
+        // block n0 + i -> stage i % kDStages: one bulk copy per token row (256 B) and lane — lanes 0-15 the K rows,
+        // 16-31 the V rows — onto the stage's barrier; the copy engine does the moving, the warp only waits
+        auto load = [&](uint32_t i) {
+            const uint32_t stg = i % kDStages, dst = tiles + stg * 2u * kTileBytes, bar = my_bar + 8u * stg;
+            if (lane == 0) mbar_expect_tx(bar, 2u * 16u * 256u);
+            __syncwarp();
+            const uint4 *src = (lane < 16 ? kbase : vbase) + (size_t)i * 256u + (lane & 15u) * 16u;
+            bulk_g2s(dst + (lane >> 4) * kTileBytes + (lane & 15u) * kTilePitch, src, 256u, bar);
         };
         AttnState st;
         attn_begin(st, a.q + ((size_t)b * a.H + h) * a.G * 128u, a.G, lane);
-        load(0);
+#pragma unroll
+        for (uint32_t i = 0; i + 1 < kDStages; ++i)
+            if (i < nb) load(i);
         for (uint32_t i = 0; i < nb; ++i) {
-            if (i + 1 < nb) {
-                load(i + 1);
-                asm volatile("cp.async.wait_group 1;" ::: "memory");
-            } else {
-                asm volatile("cp.async.wait_group 0;" ::: "memory");
+            if (i + kDStages - 1 < nb) load(i + kDStages - 1);                // into the stage freed by block i - 1
+            const uint32_t stg = i % kDStages;
+            if (!mbar_wait_warp(my_bar + 8u * stg, (phases >> stg) & 1u)) {        // never expected: report once, drop the rest of the piece
+                if (lane == 0) raise_status(a.ctl, SPECKV_ST_TIMEOUT, s_blk[b] * 2u * a.H);
+                break;
             }
-            __syncwarp();
-            const uint32_t t = tiles + (i & 1u) * 2u * kTileBytes;
+            phases ^= 1u << stg;
+            const uint32_t t = tiles + stg * 2u * kTileBytes;
             attn_block(st, t, t + kTileBytes, 16u * (n0 + i), len, lane);
-            __syncwarp();                                                     // the stage is refilled two blocks later
+            __syncwarp();                                                     // the stage is refilled by the next iteration's load
         }
         attn_end(st, a.partial + (size_t)(w + b * a.H + h) * kPartialFloats, lane);
         advance(sh, s_blk, a.B, a.H, nb);
@@ -476,7 +477,7 @@ cudaError_t launch_attend(const AttendArgs &a, bool fused, int n_sm, cudaStream_
         n_warps = grid * kFWarps;
         attend_fused_kernel<<<grid, kFWarps * 32, smem, stream>>>(a);
     } else {
-        const size_t smem = (size_t)kDWarps * 4 * kTileBytes + prefix_smem(a.B);
+        const size_t smem = (size_t)kDWarps * kDStages * 2 * kTileBytes + kDWarps * kDStages * 8 + prefix_smem(a.B);
         e = cudaFuncSetAttribute(attend_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         uint32_t grid = min((uint32_t)n_sm * 3u, attend_max_warps() / kDWarps);
