@@ -218,8 +218,9 @@ int speckv_decompress_gather_host(speckv_ctx *ctx, uint32_t layer, const int32_t
  * every entry gets its new offset and the cursor becomes the number of 64-byte units kept.  An
  * entry whose record is not inside the pool is reported (SPECKV_ST_BAD_RECORD, index = slot) and
  * cleared.  scratch: DEVICE memory, 256-byte aligned, at least speckv_compact_scratch_bytes(ctx)
- * bytes (pool_bytes + 4 bytes per slot + a little), contents undefined afterwards.  Prefetch
- * residency tags stay valid (they name blocks, not offsets).
+ * bytes (pool_bytes + 8 bytes per slot + one bit per 64 bytes of pool + a little), contents undefined
+ * afterwards.  Pool bytes behind the last record kept are unspecified.  Prefetch residency tags stay valid
+ * (they name blocks, not offsets).
  *
  * speckv_free_slots gives slots back (a finished request's blocks): the listed page-table entries are
  * cleared, so the slots read as never written and their records are garbage that the next speckv_compact

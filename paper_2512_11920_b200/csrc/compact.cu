@@ -2,24 +2,32 @@
 // its old record behind; this rewrites the pool so that it holds exactly the records that page-table
 // entries point at, in slot order, from granule 0 on.  Four small kernels on one stream:
 //   sizes     : one thread per slot -> granules of its record (0 if none); entries whose record is not
-//               inside the pool are reported and cleared; per-block (1,024 slots) totals
+//               inside the pool are reported and cleared; per-block (1,024 slots) totals; the granules
+//               that live records occupy are marked in a bitmap (one bit per granule of the pool)
 //   scan      : one CTA, exclusive prefix of the block totals, new cursor
-//   move      : one CTA per block: prefix inside the block, then one warp per record copies it to its
-//               new place in the scratch area and rewrites the entry
-//   copy back : scratch -> pool, as many granules as were kept
+//   move      : one CTA per block: prefix inside the block, then one warp per record.  If no marked
+//               granule lies in the record's new place, nothing that is still to be read can be
+//               overwritten there: the warp reads the whole record into registers and writes it
+//               straight to its final place.  Otherwise the record goes to the same place in the
+//               scratch area and is flagged.  Either way the entry is rewritten.
+//   copy back : one warp per flagged record: scratch -> pool
+// A record moved directly costs one read and one write, a flagged one two of each.
 #include "speckv_dev.cuh"
 
 namespace speckv {
 
 constexpr uint32_t kCBlock = 1024;      // slots per CTA
 constexpr uint32_t kCThreadsC = 256;
+constexpr uint32_t kMaxRecPieces = ((kHdrBytes + kPageBytes + kGranule - 1u) / kGranule * 4u + 31u) / 32u;   // 16-byte pieces per lane: 9
 
 struct CompactArgs {
     uint8_t *pool, *scratch;
     unsigned long long *pte;
     Ctl *ctl;
-    uint32_t *gran;                       // [n_slots] granules per slot
+    uint32_t *gran;                       // [n_slots] granules per slot; bit 31: the record waits in the scratch area
+    uint32_t *dest;                       // [n_slots] new place (granule) of a flagged record
     unsigned long long *block_base;       // [n_blocks + 1] totals, then exclusive prefixes
+    uint32_t *live;                       // [ceil(pool_gran / 32)] bit g: granule g belongs to a live record's old place
     unsigned long long n_slots, pool_gran;
     uint32_t n_blocks;
 };
@@ -53,6 +61,13 @@ __global__ void __launch_bounds__(kCThreadsC) compact_sizes_kernel(CompactArgs a
                 raise_status(a.ctl, SPECKV_ST_BAD_RECORD, (uint32_t)slot);
                 a.pte[slot] = 0ull;
                 g = 0;
+            } else {
+                const unsigned long long lo = e & 0xFFFFFFFFull, hi = lo + g;          // granules [lo, hi)
+                for (unsigned long long w = lo >> 5; w <= (hi - 1) >> 5; ++w) {
+                    const unsigned long long b0 = w << 5;
+                    const uint32_t from = lo > b0 ? (uint32_t)(lo - b0) : 0u, to = hi < b0 + 32 ? (uint32_t)(hi - b0) : 32u;
+                    atomicOr(&a.live[w], (to == 32u ? 0xFFFFFFFFu : ((1u << to) - 1u)) & ~((1u << from) - 1u));
+                }
             }
         }
         a.gran[slot] = g;
@@ -128,21 +143,55 @@ __global__ void __launch_bounds__(kCThreadsC) compact_move_kernel(CompactArgs a)
             if (lane == 0) { raise_status(a.ctl, SPECKV_ST_POOL_FULL, (uint32_t)slot); a.pte[slot] = 0ull; }
             continue;
         }
-        uint4 *dst = reinterpret_cast<uint4 *>(a.scratch + at * kGranule);
-        for (uint32_t i = lane; i < n_gran * 4u; i += 32) dst[i] = __ldg(src + i);
+        // is any granule of the new place still somebody's old place (this record's own included: another
+        // entry may share it)?
+        bool busy = false;
+        {
+            const unsigned long long lo = at, hi = at + n_gran, w = (lo >> 5) + lane;
+            if (w <= (hi - 1) >> 5) {
+                const unsigned long long b0 = w << 5;
+                const uint32_t from = lo > b0 ? (uint32_t)(lo - b0) : 0u, to = hi < b0 + 32 ? (uint32_t)(hi - b0) : 32u;
+                busy = (a.live[w] & (to == 32u ? 0xFFFFFFFFu : ((1u << to) - 1u)) & ~((1u << from) - 1u)) != 0u;
+            }
+        }
+        if (__any_sync(kFull, busy)) {
+            uint4 *dst = reinterpret_cast<uint4 *>(a.scratch + at * kGranule);
+            for (uint32_t i = lane; i < n_gran * 4u; i += 32) dst[i] = src[i];    // plain loads: this kernel also writes the pool
+            if (lane == 0) { a.gran[slot] = n_gran | 0x80000000u; a.dest[slot] = (uint32_t)at; }
+        } else {
+            uint4 buf[kMaxRecPieces];                      // the whole record (at most 4,160 bytes) in the warp's registers
+#pragma unroll
+            for (uint32_t j = 0; j < kMaxRecPieces; ++j)
+                if (j * 32u + lane < n_gran * 4u) buf[j] = src[j * 32u + lane];
+            uint4 *dst = reinterpret_cast<uint4 *>(a.pool + at * kGranule);
+#pragma unroll
+            for (uint32_t j = 0; j < kMaxRecPieces; ++j)
+                if (j * 32u + lane < n_gran * 4u) dst[j * 32u + lane] = buf[j];
+        }
         if (lane == 0) a.pte[slot] = (e & ~0xFFFFFFFFull) | at;
     }
 }
 
 __global__ void __launch_bounds__(256) compact_copy_back_kernel(CompactArgs a)
 {
-    const unsigned long long kept = a.block_base[a.n_blocks];
-    const unsigned long long n16 = (kept < a.pool_gran ? kept : a.pool_gran) * (kGranule / 16);
-    const uint4 *src = reinterpret_cast<const uint4 *>(a.scratch);
-    uint4 *dst = reinterpret_cast<uint4 *>(a.pool);
-    for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < n16;
-         i += (unsigned long long)gridDim.x * blockDim.x)
-        dst[i] = src[i];
+    const uint32_t lane = threadIdx.x & 31u;
+    const unsigned long long n_warps = (unsigned long long)gridDim.x * (blockDim.x >> 5);
+    for (unsigned long long s0 = ((unsigned long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * 32ull; s0 < a.n_slots;
+         s0 += n_warps * 32ull) {
+        // 32 slots at a time: one coalesced read of their flags, then the flagged ones in turn
+        const unsigned long long mine = s0 + lane;
+        const uint32_t g = mine < a.n_slots ? a.gran[mine] : 0u;
+        uint32_t todo = __ballot_sync(kFull, (g & 0x80000000u) != 0u);
+        while (todo) {
+            const uint32_t l = __ffs(todo) - 1u;
+            todo &= todo - 1u;
+            const uint32_t n_gran = __shfl_sync(kFull, g, l) & 0x7FFFFFFFu;
+            const uint32_t at = a.dest[s0 + l];
+            const uint4 *src = reinterpret_cast<const uint4 *>(a.scratch + (unsigned long long)at * kGranule);
+            uint4 *dst = reinterpret_cast<uint4 *>(a.pool + (unsigned long long)at * kGranule);
+            for (uint32_t i = lane; i < n_gran * 4u; i += 32) dst[i] = src[i];
+        }
+    }
 }
 
 // speckv_free_slots: one thread per list entry swaps the page-table entry for zero; what it found there
@@ -175,10 +224,13 @@ cudaError_t launch_free_slots(unsigned long long *pte, unsigned long long n_slot
     return cudaGetLastError();
 }
 
+static unsigned long long align256(unsigned long long v) { return (v + 255ull) & ~255ull; }
+
+// scratch layout: [pool_bytes] records | [n_slots] granules | [n_slots] new places | block prefixes | live bitmap
 size_t compact_scratch_bytes(unsigned long long n_slots, unsigned long long pool_bytes)
 {
     const unsigned long long n_blocks = (n_slots + kCBlock - 1) / kCBlock;
-    return (size_t)(pool_bytes + ((n_slots * 4 + 255) & ~255ull) + (n_blocks + 1) * 8);
+    return (size_t)(pool_bytes + 2 * align256(n_slots * 4) + align256((n_blocks + 1) * 8) + align256((pool_bytes / kGranule + 31) / 32 * 4));
 }
 
 cudaError_t launch_compact(uint8_t *pool, unsigned long long pool_bytes, unsigned long long *pte, unsigned long long n_slots,
@@ -186,10 +238,16 @@ cudaError_t launch_compact(uint8_t *pool, unsigned long long pool_bytes, unsigne
 {
     CompactArgs a;
     a.pool = pool; a.scratch = scratch; a.pte = pte; a.ctl = ctl;
-    a.gran = reinterpret_cast<uint32_t *>(scratch + pool_bytes);
-    a.block_base = reinterpret_cast<unsigned long long *>(scratch + pool_bytes + ((n_slots * 4 + 255) & ~255ull));
+    const unsigned long long n_blocks = (n_slots + kCBlock - 1) / kCBlock;
+    uint8_t *p = scratch + pool_bytes;
+    a.gran = reinterpret_cast<uint32_t *>(p); p += align256(n_slots * 4);
+    a.dest = reinterpret_cast<uint32_t *>(p); p += align256(n_slots * 4);
+    a.block_base = reinterpret_cast<unsigned long long *>(p); p += align256((n_blocks + 1) * 8);
+    a.live = reinterpret_cast<uint32_t *>(p);
     a.n_slots = n_slots; a.pool_gran = pool_bytes / kGranule;
-    a.n_blocks = (uint32_t)((n_slots + kCBlock - 1) / kCBlock);
+    a.n_blocks = (uint32_t)n_blocks;
+    cudaError_t e = cudaMemsetAsync(a.live, 0, (size_t)((a.pool_gran + 31) / 32 * 4), stream);
+    if (e != cudaSuccess) return e;
     compact_sizes_kernel<<<a.n_blocks, kCThreadsC, 0, stream>>>(a);
     compact_scan_kernel<<<1, 1024, 0, stream>>>(a);
     compact_move_kernel<<<a.n_blocks, kCThreadsC, 0, stream>>>(a);

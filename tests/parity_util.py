@@ -165,7 +165,9 @@ class Pair:
         return self._attend_check(out.cpu().numpy(), want, self._vmax(d, seq_lens, tpad, tok), n_q_heads // H, "decompress_attend")
 
     # ---- state comparison ----------------------------------------------------------------
-    def check_state(self):
+    def check_state(self, pool_defined_bytes=None):
+        """pool_defined_bytes: compare the pool only up to there (after a compaction whose copies did not all fit,
+        the bytes behind the last copy that did are unspecified)."""
         cur = self.gpu.cursor()
         assert cur == self.cpu.cursor.value, f"cursor {cur} != {self.cpu.cursor.value}"
         pte = self.gpu.pte_view().cpu().numpy().view(np.uint64)
@@ -179,6 +181,8 @@ class Pair:
         total = self.cpu.cfg.pool_bytes
         used = min(cur * 64, total)
         upto = total if total <= (1 << 28) else min(total, used + (64 << 20))
+        if pool_defined_bytes is not None:
+            upto = used = min(upto, pool_defined_bytes)
         pool = self.gpu.pool_view(upto).cpu().numpy()
         if not np.array_equal(pool, self.cpu.pool[:upto]):
             bad = np.nonzero(pool != self.cpu.pool[:upto])[0]

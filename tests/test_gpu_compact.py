@@ -72,7 +72,7 @@ def test_entries_sharing_records_overflow_the_pool():
     for pte in (pr.cpu.pte, pr.gpu.pte_view().view(pr.torch.int64)):
         pte[1] = int(pr.cpu.pte[0]); pte[3] = int(pr.cpu.pte[2])
     pr.compact()
-    pr.check_state()
+    pr.check_state(pool_defined_bytes=10 * 64)                                     # two copies of 5 granules fitted
     st = pr.gpu.status()
     assert pr.gpu.cursor() == 20 and st["count"][O.ST_POOL_FULL] == 2 and st["first"][O.ST_POOL_FULL] == 2
     pr.close()
@@ -89,7 +89,8 @@ def test_entries_sharing_records_overflow_the_pool():
     gpte[pr.torch.from_numpy(free).to(pr.dev)] = gpte[pr.torch.from_numpy(slots.astype(np.int64)).to(pr.dev)]
     pr.cpu.pte[free] = pr.cpu.pte[slots]
     pr.compact()
-    pr.check_state()
+    live_end = max((int(e) & 0xFFFFFFFF) + (((int(e) >> 32) & 0xFFFF) + 63) // 64 for e in pr.cpu.pte if (int(e) >> 56) & 1)
+    pr.check_state(pool_defined_bytes=live_end * 64)
     st = pr.gpu.status()
     assert pr.gpu.cursor() == 2 * used and 0 < st["count"][O.ST_POOL_FULL] < len(slots)
     live = int((pr.cpu.pte >> 56 & 1).sum())
@@ -120,4 +121,27 @@ def test_free_slots_then_compaction_reclaims_a_finished_sequence():
     pr.compact()
     pr.check_state()
     assert pr.gpu.cursor() == before - gran
+    pr.close()
+
+
+def test_compaction_moves_records_straight_into_vacated_space():
+    """Every slot written twice: the log is [old versions][live versions], so every record's new place lies in
+    garbage and no live record is in the way — the records are moved without the detour through the scratch
+    area (which the test leaves poisoned: nothing of it may reach the pool)."""
+    w = workloads.llama70b(seed=23, n_layers=2, batch=4, seq=448)
+    pr = Pair.for_workload(w, pool_bytes=w.n_slots * (4160 + 2368))
+    slots = np.concatenate([w.layer_slots(0), w.layer_slots(1)])
+    pages = w.gen_pages(slots)
+    pr.compress(pages, np.arange(len(slots)), slots, 0)                             # old versions: raw, larger than what replaces them
+    pr.compress(pages, np.arange(len(slots)), slots, 3)                             # live versions behind them
+    half = pr.gpu.cursor()
+    pr.cpu.compact()
+    scratch = pr.torch.full((pr.gpu.compact_scratch_bytes(),), 0xA5, dtype=pr.torch.uint8, device=pr.dev)
+    pr.gpu.compact(scratch)
+    live_end = pr.cpu.cursor.value
+    assert live_end < half - live_end                                               # the live records fit into the garbage in front
+    pr.check_state(pool_defined_bytes=live_end * 64)
+    assert bool((scratch[:live_end * 64] == 0xA5).all()), "a record went through the scratch area"
+    for layer in range(2):
+        pr.gather(layer, w.block_table, w.seq_lens, w.dst_tok_off())
     pr.close()
