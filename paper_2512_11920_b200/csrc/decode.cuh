@@ -71,20 +71,16 @@ __device__ __forceinline__ bool decode_page(const uint8_t *rec, uint32_t mode, u
         uint32_t mk[8], c[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) { mk[k] = rec[kHdrBytes + k * 32 + lane]; c[k] = __popc(mk[k]); }
-        // rank of each group's first run = prefix sum of popcounts in (k, lane) order
-        uint32_t pa = c[0] | (c[1] << 10) | (c[2] << 20);
-        uint32_t pb = c[3] | (c[4] << 10) | (c[5] << 20);
-        uint32_t pc = c[6] | (c[7] << 10);
+        // rank of each group's first run = exclusive prefix sum of popcounts in (k, lane) order: within a row the
+        // exclusive sums stay below 8 * 31, so four rows share a word as byte fields; row totals by warp reduction
+        const uint32_t ea = scan_excl_bytes(c[0] + (c[1] << 8) + (c[2] << 16) + (c[3] << 24));
+        const uint32_t eb = scan_excl_bytes(c[4] + (c[5] << 8) + (c[6] << 16) + (c[7] << 24));
+        uint32_t excl[8], tot[8];
 #pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            uint32_t ta = __shfl_up_sync(kFull, pa, d), tb = __shfl_up_sync(kFull, pb, d), tc = __shfl_up_sync(kFull, pc, d);
-            if (lane >= (uint32_t)d) { pa += ta; pb += tb; pc += tc; }
+        for (int k = 0; k < 8; ++k) {
+            excl[k] = __byte_perm(k < 4 ? ea : eb, 0u, 0x4440 + (k & 3));
+            tot[k] = __reduce_add_sync(kFull, c[k]);
         }
-        uint32_t ta = __shfl_sync(kFull, pa, 31), tb = __shfl_sync(kFull, pb, 31), tc = __shfl_sync(kFull, pc, 31);
-        uint32_t incl[8] = {pa & 1023u, (pa >> 10) & 1023u, pa >> 20, pb & 1023u, (pb >> 10) & 1023u, pb >> 20,
-                            pc & 1023u, pc >> 10};
-        uint32_t tot[8] = {ta & 1023u, (ta >> 10) & 1023u, ta >> 20, tb & 1023u, (tb >> 10) & 1023u, tb >> 20,
-                           tc & 1023u, tc >> 10};
         uint32_t total = 0;
 #pragma unroll
         for (int k = 0; k < 8; ++k) total += tot[k];
@@ -94,7 +90,7 @@ __device__ __forceinline__ bool decode_page(const uint8_t *rec, uint32_t mode, u
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             // bytes [R-1, R+8) of the value stream: the run in progress, then this group's new runs
-            uint32_t A = base + incl[k] - c[k];
+            uint32_t A = base + excl[k];
             const uint32_t *w = reinterpret_cast<const uint32_t *>(rec + (A & ~3u));
             uint32_t sh = A << 3;                             // funnel shifts use the low 5 bits: 8 * (A & 3)
             uint32_t w0 = w[0], w1 = w[1], w2 = w[2];

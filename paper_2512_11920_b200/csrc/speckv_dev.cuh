@@ -92,6 +92,23 @@ __host__ __device__ inline uint32_t expand_sel(uint32_t h)
     return sel;
 }
 
+// Exclusive prefix sum over the lanes of four byte fields at once.  The caller guarantees that no
+// field's sum over any 31 lanes reaches 256.  The shuffle's own "source lane exists" predicate guards
+// the additions.
+__device__ __forceinline__ uint32_t scan_excl_bytes(uint32_t v)
+{
+    uint32_t e;
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b32 t;\n\t"
+                 "shfl.sync.up.b32 %0|p, %1, 1, 0, 0xffffffff;\n\t@!p mov.b32 %0, 0;\n\t"
+                 "shfl.sync.up.b32 t|p, %0, 1, 0, 0xffffffff;\n\t@p add.u32 %0, %0, t;\n\t"
+                 "shfl.sync.up.b32 t|p, %0, 2, 0, 0xffffffff;\n\t@p add.u32 %0, %0, t;\n\t"
+                 "shfl.sync.up.b32 t|p, %0, 4, 0, 0xffffffff;\n\t@p add.u32 %0, %0, t;\n\t"
+                 "shfl.sync.up.b32 t|p, %0, 8, 0, 0xffffffff;\n\t@p add.u32 %0, %0, t;\n\t"
+                 "shfl.sync.up.b32 t|p, %0, 16, 0, 0xffffffff;\n\t@p add.u32 %0, %0, t;\n\t}"
+                 : "=&r"(e) : "r"(v));
+    return e;
+}
+
 // ---- kernel arguments and launchers ----
 
 struct CompressArgs {
