@@ -295,12 +295,12 @@ __global__ void __launch_bounds__(kFWarps * 32, 2) attend_fused_kernel(AttendArg
 {
     extern __shared__ __align__(16) uint8_t smem[];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");          // the merge kernel may be scheduled behind this grid
-    uint32_t *s_lut = reinterpret_cast<uint32_t *>(smem + kFWarps * kFWarpBytes);          // [256]
+    uint4 *s_lut = reinterpret_cast<uint4 *>(smem + kFWarps * kFWarpBytes);          // [256]
     unsigned long long *s_bar = reinterpret_cast<unsigned long long *>(s_lut + 256);      // [kFWarps][2]
     uint32_t *s_blk = reinterpret_cast<uint32_t *>(s_bar + kFWarps * 2);
     const uint32_t tid = threadIdx.x, lane = tid & 31u;
     const uint32_t warp = __shfl_sync(kFull, tid >> 5, 0);
-    s_lut[tid & 255u] = expand_sel(tid & 15u) | (expand_sel((tid >> 4) & 15u) << 16);
+    s_lut[tid & 255u] = expand_entry(tid & 255u);
     if (tid < kFWarps * 2) mbar_init(smem_u32(s_bar + tid), 1);
     mbar_init_fence();
     build_prefix(a, s_blk, tid, kFWarps * 32, a.max_blocks_per_seq);
@@ -470,7 +470,7 @@ cudaError_t launch_attend(const AttendArgs &a, bool fused, int n_sm, cudaStream_
     cudaError_t e;
     uint32_t n_warps;
     if (fused) {
-        const size_t smem = (size_t)kFWarps * kFWarpBytes + 256 * 4 + kFWarps * 2 * 8 + prefix_smem(a.B);
+        const size_t smem = (size_t)kFWarps * kFWarpBytes + 256 * 16 + kFWarps * 2 * 8 + prefix_smem(a.B);
         e = cudaFuncSetAttribute(attend_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         uint32_t grid = min((uint32_t)n_sm * 2u, attend_max_warps() / kFWarps);

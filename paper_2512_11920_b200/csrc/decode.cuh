@@ -23,6 +23,14 @@ __device__ __forceinline__ Walk decode_pte(unsigned long long e, unsigned long l
     return w;
 }
 
+// Table entry of the run expansion for a head mask m of 8 symbols: x, y = PRMT selectors of symbols 0-3 and 4-7
+// (index into "byte in progress + following run values"), z = 8 * number of heads among symbols 0-3 (how far the
+// second word's window is shifted).
+__device__ __forceinline__ uint4 expand_entry(uint32_t m)
+{
+    return make_uint4(expand_sel(m & 15u), expand_sel((m >> 4) & 15u), 8u * __popc(m & 15u), 0u);
+}
+
 // ---------------------------------------------------------------- small PTX wrappers
 
 // packed binary32 pairs: (a - b) * c with one rounding per operation and element
@@ -49,10 +57,10 @@ __device__ __forceinline__ float biased(uint32_t t) { return __uint_as_float(__b
 // Decodes the staged record (mode 1..3, with or without SPECKV_GROUPED) and hands the page out as
 // eight calls store(k, v): v = the 8 binary16 values at flat index 256*k + 8*lane (token row
 // 2*k + lane/16, channels 8*(lane%16)..).  Returns false if the record is inconsistent (nothing
-// is stored then).  `lut` = 256 words, entry m = expand_sel(m & 15) | expand_sel(m >> 4) << 16.
+// is stored then).  `lut` = 256 entries made by expand_entry().
 template <class Store>
 __device__ __forceinline__ bool decode_page(const uint8_t *rec, uint32_t mode, uint32_t payload_len, uint32_t n_runs,
-                                            float s, const uint32_t *lut, uint32_t lane, Store store)
+                                            float s, const uint4 *lut, uint32_t lane, Store store)
 {
     if (mode & SPECKV_GROUPED) {
         // one scale per group of 8 channels = per pair of lanes (l, l + 16), from the stored maximum
@@ -94,12 +102,11 @@ __device__ __forceinline__ bool decode_page(const uint8_t *rec, uint32_t mode, u
             const uint32_t *w = reinterpret_cast<const uint32_t *>(rec + (A & ~3u));
             uint32_t sh = A << 3;                             // funnel shifts use the low 5 bits: 8 * (A & 3)
             uint32_t w0 = w[0], w1 = w[1], w2 = w[2];
-            uint32_t v0 = __funnelshift_r(w0, w1, sh), v1 = __funnelshift_r(w1, w2, sh), v2 = w2 >> (sh & 31u);
-            uint32_t sel = lut[mk[k]];
-            sy[k][0] = __byte_perm(v0, v1, sel & 0xFFFFu);
-            uint32_t c0 = __popc(mk[k] & 15u) * 8u;
-            uint32_t u0 = __funnelshift_rc(v0, v1, c0), u1 = __funnelshift_rc(v1, v2, c0);
-            sy[k][1] = __byte_perm(u0, u1, sel >> 16);
+            uint32_t v0 = __funnelshift_r(w0, w1, sh), v1 = __funnelshift_r(w1, w2, sh), v2 = __funnelshift_r(w2, 0u, sh);
+            const uint4 e = lut[mk[k]];                       // selectors of the two words, 8 * (heads in the first word)
+            sy[k][0] = __byte_perm(v0, v1, e.x);
+            uint32_t u0 = __funnelshift_rc(v0, v1, e.z), u1 = __funnelshift_rc(v1, v2, e.z);
+            sy[k][1] = __byte_perm(u0, u1, e.y);
             base += tot[k];
         }
     } else {

@@ -55,7 +55,7 @@ __global__ void __launch_bounds__(kGThreads, 3) gather_kernel(GatherArgs a)
 {
     extern __shared__ __align__(16) uint8_t smem[];
     uint8_t *s_rec = smem;                                                        // [kGWarps][2][kStage]
-    uint32_t *s_lut = reinterpret_cast<uint32_t *>(smem + kGWarps * 2 * kStage);   // [256]
+    uint4 *s_lut = reinterpret_cast<uint4 *>(smem + kGWarps * 2 * kStage);   // [256]
     unsigned long long *s_bar = reinterpret_cast<unsigned long long *>(s_lut + 256);   // [kGWarps][2]
     unsigned long long *s_tok = s_bar + kGWarps * 2;                              // [B] first token row of each sequence
     uint32_t *s_pref = reinterpret_cast<uint32_t *>(s_tok + a.B);                 // [B + 1] exclusive prefix of blocks
@@ -68,7 +68,7 @@ __global__ void __launch_bounds__(kGThreads, 3) gather_kernel(GatherArgs a)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const uint32_t tid = threadIdx.x, lane = tid & 31u;
     const uint32_t warp = __shfl_sync(kFull, tid >> 5, 0);                        // warp-uniform for the compiler too
-    s_lut[tid & 255u] = expand_sel(tid & 15u) | (expand_sel((tid >> 4) & 15u) << 16);
+    s_lut[tid & 255u] = expand_entry(tid & 255u);
     if (tid < kGWarps * 2) mbar_init(smem_u32(s_bar + tid), 1);
     // blocks per sequence; a length that the block table cannot describe contributes none (reported below)
     for (uint32_t b = tid; b < a.B; b += kGThreads) {
@@ -249,7 +249,7 @@ __global__ void __launch_bounds__(kGThreads, 3) gather_kernel(GatherArgs a)
 
 static size_t gather_smem_bytes(uint32_t B)
 {
-    return (size_t)kGWarps * 2 * kStage + 256 * 4 + kGWarps * 2 * 8 + (size_t)B * 8 + ((size_t)B + 1) * 4;
+    return (size_t)kGWarps * 2 * kStage + 256 * 16 + kGWarps * 2 * 8 + (size_t)B * 8 + ((size_t)B + 1) * 4;
 }
 
 cudaError_t launch_gather(const GatherArgs &a, int n_sm, cudaStream_t stream)

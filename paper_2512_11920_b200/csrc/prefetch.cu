@@ -154,7 +154,7 @@ __global__ void __launch_bounds__(kPfThreads, 3) pf_fetch_kernel(PrefetchArgs a)
 {
     extern __shared__ __align__(16) uint8_t smem[];
     uint8_t *s_rec = smem;                                                        // [kPfWarps][2][kRecStage]
-    uint32_t *s_lut = reinterpret_cast<uint32_t *>(smem + kPfWarps * 2 * kRecStage);   // [256]
+    uint4 *s_lut = reinterpret_cast<uint4 *>(smem + kPfWarps * 2 * kRecStage);   // [256]
     unsigned long long *s_bar = reinterpret_cast<unsigned long long *>(s_lut + 256);   // [kPfWarps][2]
     uint32_t *s_cnt = reinterpret_cast<uint32_t *>(s_bar + kPfWarps * 2);         // [B + 1] live units before sequence b
     uint32_t *s_unit = s_cnt + a.B + 1;                                           // [<= 8 B] block << 12 | sequence << 3 | unit
@@ -162,7 +162,7 @@ __global__ void __launch_bounds__(kPfThreads, 3) pf_fetch_kernel(PrefetchArgs a)
     const uint32_t tid = threadIdx.x, lane = tid & 31u;
     const uint32_t warp = __shfl_sync(kFull, tid >> 5, 0);
     const uint32_t back = a.back, twoH = 2u * a.H;
-    s_lut[tid & 255u] = expand_sel(tid & 15u) | (expand_sel((tid >> 4) & 15u) << 16);
+    s_lut[tid & 255u] = expand_entry(tid & 255u);
     if (tid < kPfWarps * 2) mbar_init(smem_u32(s_bar + tid), 1);
     asm volatile("griddepcontrol.wait;" ::: "memory");                            // the plan's `where`, tags and fill masks
     // live units of each sequence: reads that missed (where = -1), slots transferred (fill bit)
@@ -300,7 +300,7 @@ __global__ void __launch_bounds__(kPfThreads, 3) pf_fetch_kernel(PrefetchArgs a)
 
 static size_t pf_fetch_smem(uint32_t B)
 {
-    return (size_t)kPfWarps * 2 * kRecStage + 256 * 4 + kPfWarps * 2 * 8 + ((size_t)B + 1) * 4 + (size_t)B * kPfUnits * 4;
+    return (size_t)kPfWarps * 2 * kRecStage + 256 * 16 + kPfWarps * 2 * 8 + ((size_t)B + 1) * 4 + (size_t)B * kPfUnits * 4;
 }
 
 cudaError_t launch_prefetch_step(const PrefetchArgs &a, int n_sm, cudaStream_t stream)
