@@ -36,8 +36,8 @@ PAGE = 4096
 # DRAM bytes per page (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture, divided by the
 # pages of that launch; see profiles/), valid only for the kernel sources they were captured from.
 NCU_TRAFFIC = {
-    "speckv_compress": {"bytes_per_page": 6287.8, "sources": ["compress.cu", "async_ptx.cuh", "speckv_dev.cuh"], "sha1": "2e5b669abd1b0b87a8f66be7de57fbec6334116c"},
-    "speckv_decompress_gather": {"bytes_per_page": 5590.8, "sources": ["gather.cu", "decode.cuh", "async_ptx.cuh", "speckv_dev.cuh"], "sha1": "4ce82275c9cb73b2ab03f24be9742c22bc575ea7"},
+    "speckv_compress": {"bytes_per_page": 6291.3, "sources": ["compress.cu", "async_ptx.cuh", "speckv_dev.cuh"], "sha1": "4186d566e6b25b3f549b206c0aac3e1138572dc4"},
+    "speckv_decompress_gather": {"bytes_per_page": 5586.7, "sources": ["gather.cu", "decode.cuh", "async_ptx.cuh", "speckv_dev.cuh"], "sha1": "922d504b5c3e59d79165ee7f9d49e1dd53700b35"},
 }
 
 
