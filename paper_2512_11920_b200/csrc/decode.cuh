@@ -120,24 +120,34 @@ __device__ __forceinline__ bool decode_page(const uint8_t *rec, uint32_t mode, u
 #pragma unroll
         for (int k = 0; k < 8; ++k) cb[k] = 0;
     } else {
-        // running sum of the deltas along each token row (16 lanes), modulo 256: group totals by
-        // byte dot products, then a byte-packed segmented scan over the 16 lanes of a row
-        uint32_t tlo = 0, thi = 0;
+        // Running sum of the deltas along each token row (16 lanes).  Only the sums' low bytes matter (mod 256),
+        // but a group total is at most 8 * 255 and a row has 16 lanes, so whole sums fit 16-bit fields: two groups
+        // per word, plain additions, no carries between fields.  Segmented inclusive scan over the 16 lanes of a
+        // row, then exclusive = inclusive - own, plus 128 (the low byte of every running sum is then q + 128).
+        uint32_t p[4];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            uint32_t t = __dp4a(sy[k][1], 0x01010101u, __dp4a(sy[k][0], 0x01010101u, 0u));
-            if (k < 4) tlo = __byte_perm(tlo, t, 0x3210 ^ ((4u ^ k) << (4 * k)));
-            else thi = __byte_perm(thi, t, 0x3210 ^ ((4u ^ (k - 4)) << (4 * (k - 4))));
+        for (int k = 0; k < 8; k += 2) {
+            const uint32_t t0 = __dp4a(sy[k][1], 0x01010101u, __dp4a(sy[k][0], 0x01010101u, 0u));
+            const uint32_t t1 = __dp4a(sy[k + 1][1], 0x01010101u, __dp4a(sy[k + 1][0], 0x01010101u, 0u));
+            p[k / 2] = t0 + (t1 << 16);
         }
-        uint32_t ilo = tlo, ihi = thi;
+        uint32_t inc[4] = {p[0], p[1], p[2], p[3]};
 #pragma unroll
         for (int d = 1; d < 16; d <<= 1) {
-            uint32_t a = __shfl_up_sync(kFull, ilo, d, 16), b = __shfl_up_sync(kFull, ihi, d, 16);
-            if ((lane & 15u) >= (uint32_t)d) { ilo = badd4(ilo, a); ihi = badd4(ihi, b); }
-        }
-        uint32_t elo = bsub4(ilo, tlo) ^ 0x80808080u, ehi = bsub4(ihi, thi) ^ 0x80808080u;   // exclusive carry + 128
+            const bool take = (lane & 15u) >= (uint32_t)d;
 #pragma unroll
-        for (int k = 0; k < 8; ++k) cb[k] = __byte_perm((k < 4) ? elo : ehi, 0u, 0x4440 + (k & 3));
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t up = __shfl_up_sync(kFull, inc[j], d, 16);
+                if (take) inc[j] += up;
+            }
+        }
+        // cb[k]: anything whose low byte is (exclusive sum + 128) mod 256 — the bits above are never looked at
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t e = inc[j] - p[j] + 0x00800080u;
+            cb[2 * j] = e;
+            cb[2 * j + 1] = e >> 16;
+        }
     }
     const float negb = -8388736.0f;   // -(2^23 + 128)
 #pragma unroll
