@@ -429,3 +429,58 @@ def test_sequences_longer_than_the_block_table_are_reported_and_left_out():
     pr._attend_check(out.cpu().numpy(), want, pr._vmax(d, valid, tpad, tok), 2, "decompress_attend")
     pr.check_state()
     pr.close()
+
+
+def test_reads_on_one_stream_while_another_layer_is_compressed_on_a_second():
+    """The header allows reading calls to run at the same time as a compress call whose slots they do not read
+    (the compressor only appends behind the cursor and writes its own slots' entries).  Layer 0 is fetched and
+    attended on one stream while layers 1..3 are compressed on another, with no ordering between the streams;
+    afterwards everything equals the oracle's state, and every fetch of layer 0 equals the oracle's pages."""
+    import torch
+    w = workloads.llama70b(seed=41, n_layers=4, batch=4, seq=1024)
+    pr = Pair.for_workload(w)
+    slots0 = w.layer_slots(0)
+    pr.compress(w.gen_pages(slots0), np.arange(len(slots0)), slots0, 3)
+    want = np.zeros(w.demand_tokens() * 2 * w.n_kv_heads * 128, np.uint16)
+    l2 = np.zeros(w.batch * 4 * 2 * w.n_kv_heads * 2048, np.uint16)
+    pr.cpu.decompress_gather(0, w.block_table, w.seq_lens, w.dst_tok_off(), None, want, l2)
+    want_t = torch.from_numpy(want.view(np.int16)).cuda()
+    bt, lens, tok = pr.t(w.block_table), pr.t(w.seq_lens), pr.t(w.dst_tok_off())
+    srcs = [(pr.t(w.gen_pages(w.layer_slots(l))), pr.t(np.arange(w.pages_per_layer, dtype=np.uint32)), pr.t(w.layer_slots(l))) for l in (1, 2, 3)]
+    writer, reader = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    outs = [torch.empty_like(want_t) for _ in range(12)]
+    with torch.cuda.stream(writer):
+        for src, idx, slots in srcs:
+            pr.gpu.compress(src, idx, slots, 3)
+    with torch.cuda.stream(reader):
+        for o in outs:
+            pr.gpu.decompress_gather(0, bt, lens, tok, o)
+    torch.cuda.synchronize()
+    for i, o in enumerate(outs):
+        assert torch.equal(o, want_t), f"fetch {i} of layer 0 differs while other layers were being compressed"
+    for l in (1, 2, 3):                                                            # the oracle catches up
+        slots = w.layer_slots(l)
+        pr.cpu.compress(w.gen_pages(slots), np.arange(len(slots), dtype=np.uint32), slots, 3)
+    for _ in outs[1:]:                                                             # its counters count twelve fetches too (one was made above)
+        pr.cpu.decompress_gather(0, w.block_table, w.seq_lens, w.dst_tok_off(), None, want.copy(), l2)
+    pr.check_state()
+    pr.close()
+
+
+def test_gathers_with_chaining_switched_off_give_the_same_pages():
+    import torch
+    w = workloads.llama70b(seed=8, n_layers=2, batch=4, seq=448)
+    pr = Pair.for_workload(w)
+    for layer in range(2):
+        slots = w.layer_slots(layer)
+        pr.compress(w.gen_pages(slots), np.arange(len(slots)), slots, 3)
+    pr.gpu.set_gather_chaining(False)
+    for rep in range(3):
+        for layer in range(2):
+            pr.gather(layer, w.block_table, w.seq_lens, w.dst_tok_off())
+    pr.gpu.set_gather_chaining(True)
+    for layer in range(2):
+        pr.gather(layer, w.block_table, w.seq_lens, w.dst_tok_off())
+    pr.check_state()
+    pr.close()

@@ -75,3 +75,37 @@ def test_static_entry_point_matches_context_compress_on_two_calls():
     with pytest.raises(SpeckvError, match="too many pages"):
         compress_static(torch.zeros(2048, dtype=torch.int16, device=dev), big, big, 3, pool, pte, ctl)
     ref.close()
+
+
+def test_static_entry_point_at_its_largest_size():
+    """SPECKV_STATIC_MAX_PAGES pages in one call (2 GiB of K/V, 26,215 tiles of the fixed scratch): the same log,
+    table and cursor as the context-based call; then, as a raw call (32,768 tiles of 16 pages: the whole array)."""
+    import torch
+    from kvgen import device as gen_device, workloads
+    from paper_2512_11920_b200 import Context, compress_static, STATIC_MAX_PAGES
+    if torch.cuda.mem_get_info()[0] < 12 << 30:
+        pytest.skip("needs 12 GiB of free device memory")
+    w = workloads.llama70b(seed=2, n_layers=8)                                  # 65,536 pages per layer: 8 layers = the maximum
+    n = STATIC_MAX_PAGES
+    assert w.n_slots == n
+    dev = torch.device("cuda:0")
+    src = torch.empty(n * 2048, dtype=torch.int16, device=dev)
+    scales = torch.from_numpy(w.scales).to(dev)
+    gen_device.fill(src, w.seed, 0, n, scales, w.pages_per_layer, w.n_kv_heads)
+    idx = torch.arange(n, dtype=torch.int32, device=dev)
+    for scheme, per_page in ((3, 2368), (0, 4160)):
+        pool_bytes = n * per_page
+        ref = Context(w.n_layers, w.n_kv_heads, w.blocks_per_layer, w.max_blocks_per_seq, w.batch, pool_bytes)
+        pool = torch.zeros(pool_bytes, dtype=torch.uint8, device=dev)
+        pte = torch.zeros(n, dtype=torch.int64, device=dev)
+        ctl = _ctl_block(torch)
+        ref.compress(src, idx, idx, scheme)
+        compress_static(src, idx, idx, scheme, pool, pte, ctl)
+        torch.cuda.synchronize()
+        cursor = int(ctl[:8].view(torch.int64).item())
+        assert cursor == ref.cursor() and sum(ref.status()["count"]) == 0
+        assert torch.equal(pte, ref.pte_view().view(torch.int64))
+        assert torch.equal(pool[:cursor * 64], ref.pool_view(cursor * 64))
+        ref.close()
+        del pool, pte
+        torch.cuda.empty_cache()
