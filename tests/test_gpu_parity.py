@@ -207,6 +207,37 @@ def test_decode_steps_with_prefetch_and_injected_faults():
     pr.close()
 
 
+def test_prefetched_block_rewritten_then_prefetched_again():
+    """The residency tags know (layer, block), not the record behind it: after a block's pages are rewritten, a
+    prefetch of that block is still skipped as resident until the caller clears the tag (the lazy invalidation of
+    Sec. 3.4.3 is the caller's step); after the clear the new version is fetched."""
+    w = workloads.decode_fetch(seed=8, n_layers=2, batch=3, steps=2, max_blocks_per_seq=12, len_lo=60, len_hi=150)
+    pr = Pair.for_workload(w, pool_bytes=w.n_slots * 2368 * 2)
+    for layer in range(w.n_layers):
+        slots = w.layer_slots(layer)
+        pr.compress(w.gen_pages(slots), np.arange(len(slots)), slots, 3)
+    lens = np.minimum(w.seq_lens, 40).astype(np.uint32)
+    tok = w.dst_tok_off(lens)
+    pf = np.array([(1, 3, 2)], O.PREFETCH)                                        # sequence 1, block 3 -> slot 2
+    _, first = pr.gather(1, w.block_table, lens, tok, pf)
+    assert pr.gpu.stats()["pf_issued"] == 1
+    # the block's pages get new contents (those of another block), raw this time
+    slots = w.layer_slots(1, [int(w.block_table[1, 3])])
+    other = w.layer_slots(1, [int(w.block_table[0, 0])])
+    pr.compress(w.gen_pages(other), np.arange(len(slots)), slots, 0)
+    _, again = pr.gather(1, w.block_table, lens, tok, pf)
+    assert pr.gpu.stats()["pf_skipped"] == 1 and np.all(again == 0xCDCD)          # taken for resident: nothing moved
+    t = 1 * 4 + 2
+    pr.cpu.l2_tag[t] = 0
+    pr.gpu.l2_tag_view().view(pr.torch.int64)[t] = 0
+    _, fresh = pr.gather(1, w.block_table, lens, tok, pf)
+    assert pr.gpu.stats()["pf_issued"] == 2
+    page = lambda buf: buf.reshape(-1, 2048)[(1 * 4 + 2) * 2 * w.n_kv_heads:(1 * 4 + 3) * 2 * w.n_kv_heads]
+    assert np.array_equal(page(fresh), w.gen_pages(other)) and not np.array_equal(page(fresh), page(first))
+    pr.check_state()
+    pr.close()
+
+
 def test_device_generator_matches_numpy_generator():
     import torch
     from kvgen import device
