@@ -27,7 +27,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from kvgen import workloads  # noqa: E402
+from kvgen import gen, workloads  # noqa: E402
 
 METRIC = "compress & decompress+gather GB/s (uncompressed KV)"
 PAGE = 4096
@@ -116,8 +116,7 @@ class Bench:
         self.pages = self.L * ppl
         self.src = torch.empty(self.pages * 2048, dtype=torch.int16, device=dev)
         self.scales = torch.from_numpy(w.scales).to(dev)
-        for l in range(self.L):
-            gen_device.fill(self.src[l * ppl * 2048:(l + 1) * ppl * 2048], w.seed, (layer0 + l) * ppl, ppl, self.scales, ppl, w.n_kv_heads)
+        self.fill_source()
         pool_bytes = ((self.pages * pool_page_bytes + (64 << 20)) // 64) * 64
         self.ctx = Context(self.L, w.n_kv_heads, w.blocks_per_layer, w.max_blocks_per_seq, w.batch, pool_bytes)
         # compress lists a layer's pages in physical slot order (source and page table share the numbering)
@@ -131,6 +130,17 @@ class Bench:
         self.demand_pages = w.demand_tokens() // 16 * 2 * w.n_kv_heads * self.L
         self.raw_idx = None                 # set by mixed(): the pages that take the bypass
         torch.cuda.synchronize()
+
+    def fill_source(self):
+        """Writes the workload's pages (w.data: Gaussian, or piecewise-linear rows) into the source tensor."""
+        from kvgen import device as gen_device
+        w, ppl = self.w, self.w.pages_per_layer
+        for l in range(self.L):
+            part = self.src[l * ppl * 2048:(l + 1) * ppl * 2048]
+            if w.data == "runs":
+                gen_device.fill_runs(part, w.seed, (self.layer0 + l) * ppl, ppl)
+            else:
+                gen_device.fill(part, w.seed, (self.layer0 + l) * ppl, ppl, self.scales, ppl, w.n_kv_heads)
 
     def mixed(self, fraction=0.3, seed=11):
         """Splits the page list: a seeded `fraction` of the pages is stored raw by a scheme-0 call (the share of
@@ -877,6 +887,21 @@ def main():
         if world == 1 and not args.no_cpu_baseline:
             out["mixed_raw30"]["parity"] = b.sampled_parity(n_samples=24, seed=9)
         b.raw_idx = None
+        # the codec on pages it can shrink: piecewise-linear rows (kvgen: runs_pages) whose run-length records reach
+        # the ratio the paper reports for its delta + run-length stage; same shapes, same calls, other contents
+        w.data = "runs"
+        b.fill_source()
+        out["long_runs"] = {"data": "rows piecewise linear in the channel index, a new segment per channel with probability %d/256" % gen.RUNS_P256}
+        for name, scheme in (("delta_rle", 3), ("adaptive", 4)):
+            b.scheme = scheme
+            t = timed_passes(b, passes=8, warmup=3, sample_clocks=local)
+            k = phase_figures(b, t["comp_ms"], t["gath_ms"], t["stats"], peak, t["clocks"])
+            out["long_runs"][name] = {"scheme": scheme, "kernels": k, "clocks": t["clocks"], "pages_mode": t["stats"]["pages_mode"],
+                                      "stored_ratio": b.pages * PAGE / (64.0 * t["stats"]["granules"]), "status_counts": t["status"]["count"]}
+            if world == 1 and not args.no_cpu_baseline:
+                out["long_runs"][name]["parity"] = b.sampled_parity(n_samples=16, seed=21)
+        w.data = "gaussian"
+        b.fill_source()
     b.scheme = args.scheme
     if args.consumer:
         b.step()

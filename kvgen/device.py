@@ -34,6 +34,8 @@ def _load():
         _lib.kvgen_fill.restype = C.c_int
         _lib.kvgen_fill.argtypes = [C.c_void_p, C.c_uint64, C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p, C.c_uint64,
                                     C.c_uint32, C.c_void_p]
+        _lib.kvgen_fill_runs.restype = C.c_int
+        _lib.kvgen_fill_runs.argtypes = [C.c_void_p, C.c_uint64, C.c_uint64, C.c_uint64, C.c_uint32, C.c_void_p]
     return _lib
 
 
@@ -48,3 +50,13 @@ def fill(out, seed: int, first_pid: int, n_pages: int, scales_dev, pages_per_lay
                             scales_dev.data_ptr(), pages_per_layer, n_kv_heads, torch.cuda.current_stream().cuda_stream)
     if rc:
         raise RuntimeError(f"kvgen_fill failed: {rc}")
+
+
+def fill_runs(out, seed: int, first_pid: int, n_pages: int, p256: int = gen.RUNS_P256):
+    """Writes the piecewise-linear pages [first_pid, first_pid + n_pages) of gen.runs_pages into `out`."""
+    import torch
+    assert out.is_cuda and out.is_contiguous() and out.numel() * out.element_size() >= n_pages * 4096
+    key = int(gen.stream_key(seed) ^ np.uint64(0x52554E53))
+    rc = _load().kvgen_fill_runs(out.data_ptr(), first_pid, n_pages, key, p256, torch.cuda.current_stream().cuda_stream)
+    if rc:
+        raise RuntimeError(f"kvgen_fill_runs failed: {rc}")

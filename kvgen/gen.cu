@@ -43,7 +43,47 @@ __global__ void __launch_bounds__(256) fill_kernel(uint4 *out, unsigned long lon
     }
 }
 
+// piecewise-linear rows (gen.py: runs_pages): one thread = one token row of a page, 128 sequential steps
+__global__ void __launch_bounds__(128) fill_runs_kernel(uint4 *out, unsigned long long first_pid, unsigned long long n_pages,
+                                                        unsigned long long key, unsigned int p256)
+{
+    const unsigned long long total = n_pages * 16ull;
+    for (unsigned long long t = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; t < total;
+         t += (unsigned long long)gridDim.x * blockDim.x) {
+        const unsigned long long pid = first_pid + t / 16ull;
+        const unsigned int j = (unsigned int)(t % 16ull);
+        int u = 0, slope = 0;
+        for (unsigned int i0 = 0; i0 < 128u; i0 += 8u) {
+            unsigned int w[4];
+#pragma unroll
+            for (unsigned int e = 0; e < 8u; ++e) {
+                const unsigned int i = i0 + e;
+                const unsigned long long h = mix64(key + (pid * 2048ull + j * 128u + i) * 0x9E3779B97F4A7C15ull);
+                if (i == 0u || (unsigned int)(h & 0xFFull) < p256) slope = (int)((h >> 8) % 5ull) - 2;
+                if (i == 0u)
+                    u = j == 0u ? 127 : (int)((h >> 16) % 81ull) - 40;
+                else
+                    u = max(-127, min(127, u + slope));
+                const unsigned int bits = __half_as_ushort(__float2half_rn((float)u * 0.0078125f));
+                if (e & 1u) w[e >> 1] |= bits << 16; else w[e >> 1] = bits;
+            }
+            out[t * 16ull + i0 / 8u] = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+    }
+}
+
 }  // namespace
+
+extern "C" int kvgen_fill_runs(void *out, unsigned long long first_pid, unsigned long long n_pages, unsigned long long key,
+                               unsigned int p256, void *stream)
+{
+    if (!out) return -1;
+    if (n_pages == 0) return 0;
+    unsigned long long blocks = (n_pages * 16ull + 127ull) / 128ull;
+    if (blocks > 148ull * 64ull) blocks = 148ull * 64ull;
+    fill_runs_kernel<<<(unsigned int)blocks, 128, 0, (cudaStream_t)stream>>>((uint4 *)out, first_pid, n_pages, key, p256);
+    return cudaGetLastError() == cudaSuccess ? 0 : -2;
+}
 
 extern "C" int kvgen_fill(void *out, unsigned long long first_pid, unsigned long long n_pages, unsigned long long key,
                           const float *table_dev, const float *scales_dev, unsigned long long pages_per_layer,

@@ -95,6 +95,40 @@ def channel_scales(seed: int, n_layers: int, mode: str) -> np.ndarray:
     return sc
 
 
+RUNS_P256 = 150          # a new segment starts at a channel with probability 150/256: records of ~1,276 bytes
+
+
+def runs_pages(seed: int, page_ids, p256: int = RUNS_P256) -> np.ndarray:
+    """Pages whose rows are piecewise linear in the channel index, shape [n, 2048] uint16 (binary16 patterns):
+    the stand-in for K/V whose consecutive differences repeat, the case the delta and run-length stages are for.
+
+    Element (row j, channel i) of page `pid`, all integer arithmetic:
+
+        h      = mix64(key' + (pid * 2048 + j * 128 + i) * 0x9E3779B97F4A7C15),  key' = stream_key(seed) ^ 0x52554E53
+        start  = i == 0 or (h & 0xFF) < p256               a new segment begins here
+        slope  = ((h >> 8) % 5) - 2 at a start, else the slope of the channel before
+        u      = ((h >> 16) % 81) - 40 at i == 0 (127 in row 0), else clamp(u[i-1] + slope, -127, 127)
+        value  = u / 128                                   exact in binary16; the page's largest magnitude is 127/128
+
+    so that the quantiser's bytes are the u themselves and the delta symbols are the slopes."""
+    pid = np.asarray(page_ids, dtype=np.uint64).reshape(-1)
+    key = stream_key(seed) ^ np.uint64(0x52554E53)
+    k = np.arange(PAGE_ELEMS, dtype=np.uint64)
+    with np.errstate(over="ignore"):
+        h = mix64(key + (pid[:, None] * np.uint64(PAGE_ELEMS) + k[None, :]) * _GOLDEN).reshape(pid.size, 16, 128)
+    start = (h & np.uint64(0xFF)) < np.uint64(p256)
+    start[:, :, 0] = True
+    cand = ((h >> np.uint64(8)) % np.uint64(5)).astype(np.int64) - 2
+    last = np.maximum.accumulate(np.where(start, np.arange(128)[None, None, :], 0), axis=2)
+    slope = np.take_along_axis(cand, last, axis=2)
+    u = np.empty((pid.size, 16, 128), np.int64)
+    u[:, :, 0] = ((h[:, :, 0] >> np.uint64(16)) % np.uint64(81)).astype(np.int64) - 40
+    u[:, 0, 0] = 127
+    for i in range(1, 128):
+        u[:, :, i] = np.clip(u[:, :, i - 1] + slope[:, :, i], -127, 127)
+    return (u / 128.0).astype(np.float16).reshape(pid.size, PAGE_ELEMS).view(np.uint16)
+
+
 def structured_pages(seed: int, n: int) -> np.ndarray:
     """Test-only pages with long runs: each row is made of constant-slope segments of
     geometric length (mean 8), so that consecutive differences repeat."""

@@ -34,6 +34,7 @@ class Workload:
     scales: np.ndarray              # [n_layers][2][128] float32
     steps: int = 1
     extra: dict = field(default_factory=dict)
+    data: str = "gaussian"          # page contents: "gaussian" (gen.gen_pages) or "runs" (gen.runs_pages)
 
     @property
     def pages_per_layer(self) -> int:
@@ -65,6 +66,8 @@ class Workload:
         return int((((sl.astype(np.int64) + 15) // 16) * 16).sum())
 
     def gen_pages(self, slots) -> np.ndarray:
+        if self.data == "runs":
+            return gen.runs_pages(self.seed, slots)
         return gen.gen_pages(self.seed, slots, self.scales, self.pages_per_layer, self.n_kv_heads)
 
 

@@ -249,6 +249,34 @@ def test_device_generator_matches_numpy_generator():
     assert np.array_equal(out.cpu().numpy().view(np.uint16).reshape(n, 2048), want)
 
 
+def test_piecewise_linear_pages_device_twin_and_codec_parity():
+    """The device generator of the piecewise-linear pages equals the numpy one; on those pages (records a third of
+    the page, one to eight run heads per group) every packed scheme matches the oracle and the fetch is lossless."""
+    import torch
+    from kvgen import device
+    w = workloads.llama70b(seed=23, n_layers=2, batch=3, seq=192)
+    w.data = "runs"
+    first, n = w.pages_per_layer - 21, 2 * 21 + 5                                # straddles the layer boundary
+    out = torch.empty(n * 2048, dtype=torch.int16, device="cuda")
+    device.fill_runs(out, w.seed, first, n)
+    assert np.array_equal(out.cpu().numpy().view(np.uint16).reshape(n, 2048), w.gen_pages(np.arange(first, first + n)))
+    for scheme in (3, 4, 19, 2):
+        pr = Pair.for_workload(w)
+        for layer in range(w.n_layers):
+            slots = w.layer_slots(layer)
+            pr.compress(w.gen_pages(slots), np.arange(len(slots)), slots, scheme)
+        pr.check_state()
+        if scheme != 2:
+            assert pr.gpu.stats()["pages_mode"][3] == len(w.layer_slots(0)) * 2
+        d, _ = pr.gather(1, w.block_table, w.seq_lens, w.dst_tok_off())
+        if scheme in (3, 4):                                                      # one scale per page: exactly 1/128
+            H, tpad = w.n_kv_heads, ((w.seq_lens.astype(np.int64) + 15) // 16) * 16
+            page = d[:2048]                                                       # sequence 0, K, head 0, block 0
+            slot = ((1 * w.blocks_per_layer + int(w.block_table[0, 0])) * 2 + 0) * H + 0
+            assert np.array_equal(page.reshape(16, 128), w.gen_pages([slot])[0].reshape(16, 128)[:16])
+        pr.close()
+
+
 @pytest.mark.parametrize("H,batch", [(5, 7), (40, 3), (1, 3000)])
 def test_odd_head_counts_and_many_sequences(H, batch):
     """Head counts that do not divide the warp count, and a batch long enough to need the large
