@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(256) translate_kernel(TranslateArgs a)
 
 // ---------------------------------------------------------------- the pipelined gather
 
-__global__ void __launch_bounds__(kGThreads, 3) gather_kernel(GatherArgs a)
+__global__ void __launch_bounds__(kGThreads, 4) gather_kernel(GatherArgs a)
 {
     extern __shared__ __align__(16) uint8_t smem[];
     uint8_t *s_rec = smem;                                                        // [kGWarps][2][kStage]
@@ -264,7 +264,7 @@ cudaError_t launch_gather(const GatherArgs &a, int n_sm, cudaStream_t stream)
     uint32_t m = twoH, x = kGWarps;
     while (x) { uint32_t t = m % x; m = x; x = t; }          // m = gcd(twoH, kGWarps)
     const uint32_t mult = twoH / m;
-    uint32_t grid = (uint32_t)n_sm * 3u;
+    uint32_t grid = (uint32_t)n_sm * 4u;                     // 32 warps per SM at 64 registers: measured faster than 24 at 80
     grid = grid >= mult ? grid - grid % mult : mult;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
