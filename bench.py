@@ -336,7 +336,28 @@ class Bench:
             checked += 1
         if not same or sum(status["count"]) or sum(stats["pages_mode"]) != self.pages or stats["pages_decoded"] != self.demand_pages:
             raise RuntimeError(f"end-to-end step inconsistent: {stats} {status} host copies equal: {same}")
+        # what the host link gives to plain copies between the same buffers, both directions at once (no kernels):
+        # the bound of this leg
+        n_link = min(h_in.numel(), h_out.numel(), self.src.numel(), self.dst.numel(), 1 << 30)
+        link_ms = []
+        for _ in range(3):
+            torch.cuda.synchronize()
+            e0.record(main)
+            up.wait_event(e0)
+            down.wait_event(e0)
+            with torch.cuda.stream(up):
+                self.src[:n_link].copy_(h_in[:n_link], non_blocking=True)
+            with torch.cuda.stream(down):
+                h_out[:n_link].copy_(self.dst[:n_link], non_blocking=True)
+            main.wait_stream(up)
+            main.wait_stream(down)
+            e1.record(main)
+            torch.cuda.synchronize()
+            link_ms.append(e0.elapsed_time(e1))
+        link_gbs = 2 * n_link * 2 / (min(link_ms[1:]) * 1e-3) / 1e9
+        self.fill_source()                                   # the copy above overwrote the head of the source
         return {"ms_per_step": ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": steps, "warmup": warmup,
+                "link_gbs_plain_copies": link_gbs, "frac_of_link": (h2d + d2h) / (ms * 1e-3) / 1e9 / link_gbs,
                 "host_buffers": "one pinned copy of the whole cache each way" if ring == L else f"a ring of {ring} layers, recycled",
                 "layers_compared_with_device": checked}
 
