@@ -100,3 +100,63 @@ def one_case(seed):
 def test_random_call_sequences_match_the_oracle(seed0):
     for seed in range(seed0, seed0 + 8):
         one_case(seed)
+
+
+# ---- the attention consumers on random caches: lengths down to zero, 1-8 query heads per KV head, sharp and flat
+# softmax, rewritten and freed pages, an unmapped block
+
+def pages_for(rng, w, slots):
+    kind = rng.integers(3)
+    if kind == 0:
+        p = w.gen_pages(slots)
+    elif kind == 1:
+        p = gen.runs_pages(int(rng.integers(1 << 30)), slots, int(rng.integers(10, 250)))
+    else:
+        p = w.gen_pages(slots).copy()
+        p[rng.random(p.shape) < rng.uniform(0.3, 0.95)] = 0
+    return p
+
+
+def one_attention_case(seed):
+    rng = np.random.default_rng(seed)
+    n_layers, batch = int(rng.integers(1, 3)), int(rng.integers(1, 6))
+    if rng.integers(2):
+        mb = int(rng.integers(2, 12))
+        w = workloads.decode_fetch(seed=seed, n_layers=n_layers, batch=batch, steps=3, max_blocks_per_seq=mb, len_lo=1, len_hi=16 * mb)
+        w.seq_lens = rng.integers(1, 16 * mb + 1, size=batch).astype(np.uint32)
+    else:
+        seq = 16 * int(rng.integers(1, 40))
+        w = workloads.llama70b(seed=seed, n_layers=n_layers, batch=batch, seq=seq)
+        w.seq_lens = rng.integers(1, seq + 1, size=batch).astype(np.uint32)
+    pr = Pair.for_workload(w, pool_bytes=w.n_slots * 4160 * 2)
+    for layer in range(w.n_layers):
+        slots = w.layer_slots(layer)
+        pr.compress(pages_for(rng, w, slots), np.arange(len(slots)), slots, int(rng.choice([0, 1, 2, 3, 4, 17, 18, 19, 20])))
+    if rng.integers(2):
+        layer = int(rng.integers(w.n_layers)); slots = w.layer_slots(layer)
+        take = rng.permutation(len(slots))[: int(rng.integers(1, len(slots) + 1))]
+        pr.compress(pages_for(rng, w, slots), take, slots[take], int(rng.choice([0, 1, 2, 3, 4, 19])))
+    if rng.integers(3) == 0:
+        slots = w.layer_slots(int(rng.integers(w.n_layers)))
+        pr.free_slots(slots[rng.permutation(len(slots))[: int(rng.integers(1, 6))]])
+    bt = w.block_table.copy()
+    if rng.integers(4) == 0:
+        bt[int(rng.integers(batch)), 0] = -1
+    for _ in range(int(rng.integers(1, 4))):
+        layer = int(rng.integers(w.n_layers))
+        G = int(rng.choice([1, 2, 3, 4, 8]))
+        lens = rng.integers(0, w.seq_lens + 1).astype(np.uint32)
+        if not lens.any():
+            lens[0] = 1
+        q = (rng.standard_normal((batch, w.n_kv_heads * G, 128)) * rng.choice([0.3, 1.0, 6.0])).astype(np.float16).view(np.uint16)
+        if rng.integers(2):
+            pr.attend_fused(layer, bt, lens, q, w.n_kv_heads * G)
+        else:
+            pr.attend_dense(layer, bt, lens, q, w.n_kv_heads * G)
+    pr.check_state()
+    pr.close()
+
+
+def test_random_attention_calls_match_the_oracle():
+    for seed in range(400, 440):
+        one_attention_case(seed)
